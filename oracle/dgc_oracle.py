@@ -1,0 +1,183 @@
+"""ctypes access to the CPU oracle (oracle/dgc_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: tests, the smoke check and the benchmark's CPU
+baseline may import this module; the CUDA library and its Python binding must
+not.  It marshals numpy arrays to the C functions and holds no arithmetic of
+the method itself.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dgc_oracle.cpp")
+_LIB = os.path.join(_HERE, "libdgc_oracle.so")
+
+_i64p = ctypes.POINTER(ctypes.c_int64)
+_i32p = ctypes.POINTER(ctypes.c_int32)
+_f32p = ctypes.POINTER(ctypes.c_float)
+_f64p = ctypes.POINTER(ctypes.c_double)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (single thread, no FMA contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fPIC", "-shared",
+               "-Wall", "-Wextra", "-o", _LIB, _SRC]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        L.dgc_oracle_topk_count.restype = ctypes.c_int64
+        L.dgc_oracle_topk_count.argtypes = [ctypes.c_int64, ctypes.c_double]
+        L.dgc_oracle_warmup_sparsity.restype = ctypes.c_double
+        L.dgc_oracle_warmup_sparsity.argtypes = [ctypes.c_int32]
+        L.dgc_oracle_clip_coef.restype = None
+        L.dgc_oracle_clip_coef.argtypes = [ctypes.c_int32, _i64p, _i64p, _f32p, ctypes.c_double,
+                                           ctypes.c_int32, _f64p, _f32p]
+        L.dgc_oracle_momentum_correction.restype = None
+        L.dgc_oracle_momentum_correction.argtypes = [ctypes.c_int32, _i64p, _i64p, _f32p, _f32p,
+                                                     _f32p, ctypes.c_float, ctypes.c_float]
+        L.dgc_oracle_select_topk.restype = None
+        L.dgc_oracle_select_topk.argtypes = [ctypes.c_int64, _f32p, ctypes.c_int64, _i64p,
+                                             ctypes.c_int32]
+        L.dgc_oracle_compress.restype = None
+        L.dgc_oracle_compress.argtypes = [ctypes.c_int32, _i64p, _i64p, _i64p, _i64p, _f32p, _f32p,
+                                          _f32p, ctypes.c_float, ctypes.c_double, ctypes.c_int32,
+                                          ctypes.c_int32, ctypes.c_float, ctypes.c_int32, _i32p,
+                                          _f32p, _f64p, _f32p]
+        L.dgc_oracle_decode_accumulate.restype = None
+        L.dgc_oracle_decode_accumulate.argtypes = [ctypes.c_int32, ctypes.POINTER(_i32p),
+                                                   ctypes.POINTER(_f32p), _i64p, _f32p,
+                                                   ctypes.c_int64]
+        L.dgc_oracle_apply_sgd.restype = None
+        L.dgc_oracle_apply_sgd.argtypes = [_f32p, _f32p, ctypes.c_int64, ctypes.c_float]
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray, typ):
+    return a.ctypes.data_as(typ)
+
+
+def _chk(a: np.ndarray, dtype) -> np.ndarray:
+    assert a.dtype == dtype and a.flags["C_CONTIGUOUS"], (a.dtype, dtype)
+    return a
+
+
+def topk_count(n: int, sparsity: float) -> int:
+    return int(lib().dgc_oracle_topk_count(int(n), float(sparsity)))
+
+
+def warmup_sparsity(stage: int) -> float:
+    return float(lib().dgc_oracle_warmup_sparsity(int(stage)))
+
+
+def clip_coef(offset, numel, g, clip_threshold: float, num_workers: int):
+    offset = np.ascontiguousarray(offset, dtype=np.int64)
+    numel = np.ascontiguousarray(numel, dtype=np.int64)
+    norm = ctypes.c_double()
+    coef = ctypes.c_float()
+    lib().dgc_oracle_clip_coef(len(numel), _p(offset, _i64p), _p(numel, _i64p),
+                               _p(_chk(g, np.float32), _f32p), float(clip_threshold),
+                               int(num_workers), ctypes.byref(norm), ctypes.byref(coef))
+    return norm.value, np.float32(coef.value)
+
+
+def momentum_correction(offset, numel, u, v, g, momentum: float, coef: float) -> None:
+    offset = np.ascontiguousarray(offset, dtype=np.int64)
+    numel = np.ascontiguousarray(numel, dtype=np.int64)
+    lib().dgc_oracle_momentum_correction(len(numel), _p(offset, _i64p), _p(numel, _i64p),
+                                         _p(_chk(u, np.float32), _f32p),
+                                         _p(_chk(v, np.float32), _f32p),
+                                         _p(_chk(g, np.float32), _f32p),
+                                         ctypes.c_float(momentum), ctypes.c_float(coef))
+
+
+def select_topk(v: np.ndarray, k: int, brute_force: bool = False) -> np.ndarray:
+    v = _chk(v, np.float32)
+    sel = np.empty(k, dtype=np.int64)
+    lib().dgc_oracle_select_topk(v.size, _p(v, _f32p), int(k), _p(sel, _i64p), int(brute_force))
+    return sel
+
+
+@dataclass
+class CompressResult:
+    idx: np.ndarray      # int32, index into the arena, ascending per tensor
+    val: np.ndarray      # float32
+    norm: float          # L2 norm of the whole gradient set (fp64)
+    coef: np.float32     # clip coefficient that was applied
+
+
+class Worker:
+    """State of one worker (u, v) plus the segment table of its gradient set."""
+
+    def __init__(self, offset, numel, arena_len: int, num_workers: int, momentum: float,
+                 clip_threshold: float, sparsity: float):
+        self.offset = np.ascontiguousarray(offset, dtype=np.int64)
+        self.numel = np.ascontiguousarray(numel, dtype=np.int64)
+        self.arena_len = int(arena_len)
+        self.num_workers = int(num_workers)
+        self.momentum = float(momentum)
+        self.clip_threshold = float(clip_threshold)
+        self.u = np.zeros(self.arena_len, dtype=np.float32)   # Algorithm 4: U <- 0
+        self.v = np.zeros(self.arena_len, dtype=np.float32)   # Algorithm 4: V <- 0
+        self.set_sparsity(sparsity)
+
+    def set_sparsity(self, sparsity: float) -> None:
+        self.sparsity = float(sparsity)
+        self.k = np.array([topk_count(n, sparsity) for n in self.numel], dtype=np.int64)
+        self.out_offset = np.zeros(len(self.k) + 1, dtype=np.int64)
+        np.cumsum(self.k, out=self.out_offset[1:])
+
+    @property
+    def nnz(self) -> int:
+        return int(self.out_offset[-1])
+
+    def compress(self, g: np.ndarray, coef_override=None, brute_force: bool = False) -> CompressResult:
+        g = _chk(g, np.float32)
+        assert g.size == self.arena_len
+        idx = np.empty(self.nnz, dtype=np.int32)
+        val = np.empty(self.nnz, dtype=np.float32)
+        norm = ctypes.c_double()
+        coef = ctypes.c_float()
+        lib().dgc_oracle_compress(
+            len(self.numel), _p(self.offset, _i64p), _p(self.numel, _i64p), _p(self.k, _i64p),
+            _p(self.out_offset, _i64p), _p(self.u, _f32p), _p(self.v, _f32p), _p(g, _f32p),
+            ctypes.c_float(self.momentum), self.clip_threshold, self.num_workers,
+            int(coef_override is not None),
+            ctypes.c_float(0.0 if coef_override is None else float(coef_override)),
+            int(brute_force), _p(idx, _i32p), _p(val, _f32p), ctypes.byref(norm),
+            ctypes.byref(coef))
+        return CompressResult(idx, val, norm.value, np.float32(coef.value))
+
+
+def decode_accumulate(idx_lists, val_lists, dense_len: int) -> np.ndarray:
+    n = len(idx_lists)
+    idx_lists = [_chk(np.ascontiguousarray(a), np.int32) for a in idx_lists]
+    val_lists = [_chk(np.ascontiguousarray(a), np.float32) for a in val_lists]
+    ip = (_i32p * n)(*[_p(a, _i32p) for a in idx_lists])
+    vp = (_f32p * n)(*[_p(a, _f32p) for a in val_lists])
+    nnz = np.array([a.size for a in idx_lists], dtype=np.int64)
+    dense = np.empty(int(dense_len), dtype=np.float32)
+    lib().dgc_oracle_decode_accumulate(n, ip, vp, _p(nnz, _i64p), _p(dense, _f32p), int(dense_len))
+    return dense
+
+
+def apply_sgd(w: np.ndarray, dense_grad: np.ndarray, lr: float) -> None:
+    w = _chk(w, np.float32)
+    dense_grad = _chk(dense_grad, np.float32)
+    assert w.size == dense_grad.size
+    lib().dgc_oracle_apply_sgd(_p(w, _f32p), _p(dense_grad, _f32p), w.size, ctypes.c_float(lr))

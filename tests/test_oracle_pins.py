@@ -1,0 +1,384 @@
+"""Pins for the CPU oracle: every check here compares the oracle against
+something other than itself -- hand-worked traces (tests/golden), closed forms
+of the paper's equations, brute force, numpy library routines, invariants."""
+import json
+import os
+
+import numpy as np
+import pytest
+
+from oracle import dgc_oracle as O
+
+
+def _load(golden_dir, name):
+    with open(os.path.join(golden_dir, name)) as f:
+        return json.load(f)
+
+
+def _f32(x):
+    return np.asarray(x, dtype=np.float32)
+
+
+def _single(n, momentum, sparsity, clip=0.0, workers=1):
+    return O.Worker([0], [n], n, workers, momentum, clip, sparsity)
+
+
+# ------------------------------------------------------------------ hand-worked traces
+
+def test_alg4_two_iterations_trace(golden_dir):
+    G = _load(golden_dir, "alg4_two_iterations.json")
+    for brute in (False, True):
+        w = _single(G["n"], G["momentum"], G["sparsity"])
+        assert w.k.tolist() == [G["k"]]
+        for it in G["iterations"]:
+            r = w.compress(_f32(it["g"]), brute_force=brute)
+            assert r.idx.tolist() == it["sent_idx"]
+            assert r.val.tolist() == it["sent_val"]
+            assert w.u.tolist() == it["u_after"]
+            assert w.v.tolist() == it["v_after"]
+            assert r.coef == np.float32(1.0)
+
+
+def test_tie_goes_to_lower_index(golden_dir):
+    G = _load(golden_dir, "tie_rule.json")
+    for brute in (False, True):
+        w = _single(G["n"], G["momentum"], G["sparsity"])
+        assert w.k.tolist() == [G["k"]]
+        r = w.compress(_f32(G["g"]), brute_force=brute)
+        assert r.idx.tolist() == G["sent_idx"]
+        assert r.val.tolist() == G["sent_val"]
+
+
+def test_clip_345(golden_dir):
+    G = _load(golden_dir, "clip_345.json")
+    g = _f32(G["g"])
+    for c in G["cases"]:
+        norm, coef = O.clip_coef([0], [4], g, c["clip_threshold"], G["num_workers"])
+        assert norm == c["norm"]
+        assert coef == np.float32(c["coef"])
+        # s = 0 sends everything, so the sent values are the clipped gradient itself
+        w = O.Worker([0], [4], 4, G["num_workers"], 0.9, c["clip_threshold"], 0.0)
+        r = w.compress(g)
+        assert r.val.tolist() == c["gc"]
+        if c["coef"] == 1.0:
+            assert r.val.tobytes() == g.tobytes()     # identity bit for bit
+
+
+def test_decode_and_sgd(golden_dir):
+    G = _load(golden_dir, "decode_sgd.json")
+    idx = [np.asarray(w["idx"], dtype=np.int32) for w in G["workers"]]
+    val = [_f32(w["val"]) for w in G["workers"]]
+    dense = O.decode_accumulate(idx, val, G["dense_len"])
+    assert dense.tolist() == G["dense"]
+    w = _f32(G["w_before"]).copy()
+    O.apply_sgd(w, dense, G["lr"])
+    assert w.tolist() == G["w_after"]
+
+
+def test_warmup_schedule_and_k(golden_dir):
+    G = _load(golden_dir, "warmup_schedule.json")
+    assert [O.warmup_sparsity(i) for i in range(5)] == G["sparsity"]
+    assert O.warmup_sparsity(5) == -1.0 and O.warmup_sparsity(-1) == -1.0
+    assert [O.topk_count(G["n"], s) for s in G["sparsity"]] == G["k"]
+    for c in G["more_k"]:
+        assert O.topk_count(c["n"], c["sparsity"]) == c["k"], c
+
+
+# ------------------------------------------------------------------ selection vs brute force / numpy
+
+def _numpy_topk(v, k):
+    key = (v.view(np.uint32) & np.uint32(0x7FFFFFFF)).astype(np.int64)
+    order = np.argsort(-key, kind="stable")      # ties keep ascending index
+    return np.sort(order[:k])
+
+
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 31, 32, 33, 255, 1000, 4095, 4096])
+def test_selection_matches_full_sort(n):
+    rng = np.random.default_rng(n)
+    for trial in range(6):
+        if trial % 3 == 0:
+            v = rng.standard_normal(n).astype(np.float32)
+        elif trial % 3 == 1:      # heavy ties, both signs, zeros
+            v = rng.integers(-3, 4, size=n).astype(np.float32)
+        else:                     # mostly zeros
+            v = rng.standard_normal(n).astype(np.float32)
+            v[rng.random(n) < 0.9] = 0.0
+        for k in sorted({1, max(1, n // 1000), max(1, n // 4), max(1, n - 1), n}):
+            ref = _numpy_topk(v, k)
+            assert np.array_equal(O.select_topk(v, k, brute_force=True), ref)
+            assert np.array_equal(O.select_topk(v, k, brute_force=False), ref)
+
+
+def test_selection_special_values():
+    v = _f32([0.0, -0.0, np.inf, -np.inf, np.nan, 1e-45, -1e-45, 1.0])
+    # NaN first, then the two infinities by index, then 1.0, then denormals by index
+    assert O.select_topk(v, 1).tolist() == [4]
+    assert O.select_topk(v, 3).tolist() == [2, 3, 4]
+    assert O.select_topk(v, 4).tolist() == [2, 3, 4, 7]
+    assert O.select_topk(v, 5).tolist() == [2, 3, 4, 5, 7]
+    assert O.select_topk(v, 7).tolist() == [0, 2, 3, 4, 5, 6, 7]
+
+
+def test_selected_dominate_unselected():
+    rng = np.random.default_rng(7)
+    n = 50000
+    v = rng.standard_t(3, n).astype(np.float32)
+    k = O.topk_count(n, 0.999)
+    assert k == 50
+    sel = O.select_topk(v, k)
+    mask = np.zeros(n, bool)
+    mask[sel] = True
+    assert np.all(np.diff(sel) > 0)
+    assert np.abs(v[mask]).min() >= np.abs(v[~mask]).max()
+
+
+# ------------------------------------------------------------------ closed forms of Eq. 4 / Eq. 5
+
+def test_momentum_correction_closed_form_unsent():
+    """Eq. 4: an entry that is not sent for T iterations has accumulated
+    sum_t g_t * sum_{tau=0}^{T-t} m^tau.  One decoy entry with a huge gradient
+    is the top-1 pick every iteration, so entries 1.. are never sent."""
+    rng = np.random.default_rng(3)
+    n, T, m = 64, 12, 0.9
+    w = _single(n, m, 0.999)          # k = 1
+    G = rng.standard_normal((T, n)).astype(np.float32)
+    G[:, 0] = 1e6
+    for t in range(T):
+        r = w.compress(G[t].copy())
+        assert r.idx.tolist() == [0]
+    g64 = G.astype(np.float64)
+    expect_v = np.zeros(n)
+    expect_u = np.zeros(n)
+    for t in range(T):
+        geo = (1.0 - m ** (T - t)) / (1.0 - m)       # sum_{tau=0}^{T-t-1} m^tau  (t is 0-based)
+        expect_v += g64[t] * geo
+        expect_u += g64[t] * m ** (T - 1 - t)
+    np.testing.assert_allclose(w.v[1:], expect_v[1:], rtol=2e-5, atol=1e-6)
+    np.testing.assert_allclose(w.u[1:], expect_u[1:], rtol=2e-5, atol=1e-6)
+    assert w.v[0] == 0.0 and w.u[0] == 0.0
+
+
+def test_constant_gradient_geometric_sum_exact():
+    """u_t = g (1 - m^t)/(1 - m) for a constant gradient; exact for dyadic m, g."""
+    n, m = 16, 0.5
+    w = _single(n, m, 0.999)
+    g = np.full(n, 0.25, np.float32)
+    g[5] = 1024.0                      # always the one that is sent
+    for t in range(1, 9):
+        w.compress(g.copy())
+        u_expect = 0.25 * (1 - m ** t) / (1 - m)
+        v_expect = sum(0.25 * (1 - m ** i) / (1 - m) for i in range(1, t + 1))
+        assert w.u[0] == np.float32(u_expect)
+        assert w.v[0] == np.float32(v_expect)
+
+
+def test_zero_momentum_is_plain_accumulation():
+    """m = 0 reduces Algorithm 4 to Algorithm 1: v is the running sum of g."""
+    rng = np.random.default_rng(11)
+    n, T = 100, 7
+    w = _single(n, 0.0, 0.99)          # k = 1
+    G = rng.integers(-8, 9, size=(T, n)).astype(np.float32)   # small integers: exact sums
+    G[:, 3] = 1000.0
+    for t in range(T):
+        w.compress(G[t].copy())
+    expect = G.sum(axis=0)
+    expect[3] = 0
+    assert np.array_equal(w.v, expect)
+
+
+def test_sparsity_zero_is_dense_sgd():
+    """s = 0: every entry is sent every iteration, u and v end at zero, the sent
+    values are the (clipped) gradient: plain synchronous SGD (Algorithm 2)."""
+    rng = np.random.default_rng(5)
+    n = 257
+    w = _single(n, 0.9, 0.0, clip=0.0)
+    for t in range(3):
+        g = rng.standard_normal(n).astype(np.float32)
+        r = w.compress(g)
+        assert r.idx.tolist() == list(range(n))
+        assert r.val.tobytes() == g.tobytes()
+        assert not w.u.any() and not w.v.any()
+
+
+# ------------------------------------------------------------------ clipping vs numpy
+
+def test_clip_norm_matches_numpy_and_lands_on_threshold():
+    rng = np.random.default_rng(9)
+    numel = [1000, 37, 4096]
+    offset = [0, 1024, 1100]
+    arena = np.full(1100 + 4096, np.float32(np.nan))       # gaps hold NaN: must not be read
+    for o, n in zip(offset, numel):
+        arena[o:o + n] = rng.standard_normal(n).astype(np.float32)
+    flat = np.concatenate([arena[o:o + n] for o, n in zip(offset, numel)]).astype(np.float64)
+    norm, coef = O.clip_coef(offset, numel, arena, 4.0, 16)      # thr_local = 1.0
+    assert abs(norm - np.linalg.norm(flat)) <= 1e-12 * norm
+    assert abs(np.float64(coef) - 1.0 / np.linalg.norm(flat)) <= 1e-7 * coef
+    clipped = flat.astype(np.float32) * coef
+    assert abs(np.linalg.norm(clipped.astype(np.float64)) - 1.0) < 1e-6
+    # N^-1/2: four workers halve the threshold exactly
+    _, c1 = O.clip_coef(offset, numel, arena, 2.0, 1)
+    _, c4 = O.clip_coef(offset, numel, arena, 4.0, 4)
+    assert c1 == c4
+    # below threshold: untouched
+    _, c0 = O.clip_coef(offset, numel, arena, 1e6, 4)
+    assert c0 == np.float32(1.0)
+
+
+def test_clipping_happens_before_accumulation():
+    """Sec. 3.2: clip the new gradient, not the accumulated one."""
+    w = O.Worker([0], [4], 4, 1, 0.5, 1.0, 0.75)      # k = 1, thr_local = 1
+    r = w.compress(_f32([8, 0, 0, 6]))                 # norm 10 -> coef 0.1
+    assert r.coef == np.float32(0.1)
+    expect = _f32([8, 0, 0, 6]) * np.float32(0.1)
+    assert r.idx.tolist() == [0] and r.val[0] == expect[0]
+    assert w.v[3] == expect[3] and w.u[3] == expect[3]
+    r = w.compress(_f32([0, 0.5, 0, 0]))               # norm 0.5 < 1: no clip although |v| is larger
+    assert r.coef == np.float32(1.0)
+    assert r.idx.tolist() == [3]                       # v = [0, 0.5, 0, 0.6 + 0.3]
+    assert w.u[1] == np.float32(0.5) and w.v[1] == np.float32(0.5)
+
+
+# ------------------------------------------------------------------ invariants on a multi-tensor run
+
+def _run_multi(seed, numel, T, momentum, sparsity, clip, workers=4):
+    rng = np.random.default_rng(seed)
+    offset, pos = [], 0
+    for n in numel:
+        offset.append(pos)
+        pos += n + 5                      # gaps between tensors
+    arena_len = pos
+    w = O.Worker(offset, numel, arena_len, workers, momentum, clip, sparsity)
+    valid = np.zeros(arena_len, bool)
+    for o, n in zip(offset, numel):
+        valid[o:o + n] = True
+    shadow_u = np.zeros(arena_len)
+    shadow_acc = np.zeros(arena_len)
+    sent_sum = np.zeros(arena_len)
+    for t in range(T):
+        g = np.zeros(arena_len, np.float32)
+        g[valid] = (rng.standard_normal(valid.sum()) * 10.0 ** rng.uniform(-3, 0)).astype(np.float32)
+        g[~valid] = np.nan                # the oracle must never read a gap
+        u_before, v_before = w.u.copy(), w.v.copy()
+        r = w.compress(g)
+        # float64 shadow of Eq. 5 with the same coefficient and the same mask
+        gc = np.where(valid, g.astype(np.float64) * np.float64(r.coef), 0.0)
+        shadow_u = momentum * shadow_u + gc
+        shadow_acc += shadow_u
+        shadow_u[r.idx] = 0.0
+        sent_sum[r.idx] += r.val.astype(np.float64)
+        yield w, r, g, u_before, v_before, valid, shadow_acc, sent_sum
+
+
+@pytest.mark.parametrize("sparsity", [0.999, 0.984375, 0.75])
+def test_invariants_multi_tensor(sparsity):
+    numel = [64, 1, 5000, 333, 20000]
+    momentum = 0.9
+    for w, r, g, u_before, v_before, valid, shadow_acc, sent_sum in _run_multi(
+            1, numel, 8, momentum, sparsity, clip=1.0):
+        # nnz = ceil(n (1 - s)) per tensor
+        k = [max(1, int(np.ceil(n * (1 - sparsity) - 1e-9))) for n in numel]
+        assert w.k.tolist() == k
+        assert r.idx.size == sum(k)
+        # segments ascending, inside their tensor
+        for j, (o, n) in enumerate(zip(w.offset, w.numel)):
+            seg = r.idx[w.out_offset[j]:w.out_offset[j + 1]]
+            assert np.all(np.diff(seg) > 0)
+            assert seg.min() >= o and seg.max() < o + n
+        # u, v zero at sent entries; elsewhere equal to one step of Eq. 5 from the previous state
+        assert not w.u[r.idx].any() and not w.v[r.idx].any()
+        gc = (g * r.coef).astype(np.float32)
+        u_new = (np.float32(momentum) * u_before + gc).astype(np.float32)
+        v_new = (v_before + u_new).astype(np.float32)
+        unsent = valid.copy()
+        unsent[r.idx] = False
+        assert np.array_equal(w.u[unsent], u_new[unsent])
+        assert np.array_equal(w.v[unsent], v_new[unsent])
+        assert np.array_equal(r.val, v_new[r.idx])
+        # gaps never written
+        assert not w.u[~valid].any() and not w.v[~valid].any()
+        # selected dominate unselected, per tensor
+        for j, (o, n) in enumerate(zip(w.offset, w.numel)):
+            seg = r.idx[w.out_offset[j]:w.out_offset[j + 1]]
+            m = np.zeros(n, bool)
+            m[seg - o] = True
+            a = np.abs(v_new[o:o + n])
+            if (~m).any():
+                assert a[m].min() >= a[~m].max()
+        # conservation: sent so far + residual v = accumulated velocity (Eq. 5 in float64)
+        tol = 1e-5 * (np.abs(shadow_acc).max() + 1e-30)
+        np.testing.assert_allclose(sent_sum + w.v, shadow_acc, atol=tol, rtol=0)
+
+
+def test_selection_path_equals_brute_force_path_over_iterations():
+    numel = [4096, 17, 1000]
+    runs = []
+    for brute in (False, True):
+        rng = np.random.default_rng(21)
+        w = O.Worker([0, 4096, 4200], numel, 5200, 2, 0.9, 0.5, 0.99)
+        out = []
+        for t in range(6):
+            g = np.zeros(5200, np.float32)
+            g[:] = rng.integers(-4, 5, size=5200).astype(np.float32) * np.float32(0.125)
+            r = w.compress(g, brute_force=brute)
+            out.append((r.idx.copy(), r.val.copy(), w.u.copy(), w.v.copy()))
+        runs.append(out)
+    for a, b in zip(*runs):
+        for x, y in zip(a, b):
+            assert np.array_equal(x, y)
+
+
+# ------------------------------------------------------------------ decode / sgd vs numpy
+
+def test_decode_matches_numpy_add_at_in_worker_order():
+    rng = np.random.default_rng(2)
+    L, N = 10000, 5
+    idx = [np.sort(rng.choice(L, size=rng.integers(0, 400), replace=False)).astype(np.int32)
+           for _ in range(N)]
+    idx[2] = idx[0].copy()                    # full overlap between two workers
+    val = [rng.standard_normal(a.size).astype(np.float32) for a in idx]
+    dense = O.decode_accumulate(idx, val, L)
+    ref = np.zeros(L, np.float32)
+    for a, b in zip(idx, val):
+        ref[a] = ref[a] + b                   # unique indices per worker: plain fp32 adds, in order
+    assert dense.tobytes() == ref.tobytes()
+    # one worker: pure scatter; signed zero start is +0
+    one = O.decode_accumulate(idx[:1], val[:1], L)
+    ref1 = np.zeros(L, np.float32)
+    ref1[idx[0]] = val[0]
+    assert np.array_equal(one, ref1)
+    assert not np.signbit(one[np.setdiff1d(np.arange(L), idx[0])]).any()
+    # empty lists
+    z = O.decode_accumulate([np.zeros(0, np.int32)], [np.zeros(0, np.float32)], 7)
+    assert z.tolist() == [0.0] * 7
+
+
+def test_sgd_matches_numpy_two_roundings():
+    rng = np.random.default_rng(4)
+    w = rng.standard_normal(1001).astype(np.float32)
+    G = rng.standard_normal(1001).astype(np.float32)
+    lr = np.float32(0.1)
+    ref = (w - (lr * G).astype(np.float32)).astype(np.float32)
+    O.apply_sgd(w, G, float(lr))
+    assert w.tobytes() == ref.tobytes()
+
+
+def test_end_to_end_matches_dense_momentum_sgd_when_everything_is_eventually_sent():
+    """Eq. 3 vs Eq. 5: with momentum correction, what one worker has sent plus what
+    it still holds equals the dense momentum-SGD velocity sum -- as long as the
+    masking never fired on a non-zero u (here: s = 0 is excluded, so use the
+    residual form: sum of sent + v = sum_t u_t with u following the masked recurrence).
+    Checked exactly on dyadic data."""
+    n, m = 8, 0.5
+    w = _single(n, m, 0.75)
+    rng = np.random.default_rng(0)
+    acc = np.zeros(n)
+    u = np.zeros(n)
+    sent = np.zeros(n)
+    for t in range(6):
+        g = rng.integers(-4, 5, size=n).astype(np.float32)
+        r = w.compress(g.copy())
+        u = m * u + g
+        acc += u
+        u[r.idx] = 0
+        sent[r.idx] += r.val
+        assert np.array_equal(sent + w.v, acc)
