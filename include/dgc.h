@@ -1,0 +1,187 @@
+/*
+ * dgc.h -- C ABI of the B200-native Deep Gradient Compression hot path.
+ *
+ * One `dgc_state` is one worker ("node k" of Algorithm 4, Appendix D): it owns
+ * the two accumulators U^k and V^k of that algorithm for a whole gradient set
+ * (tensors j = 0..M laid out in one fp32 arena) and compresses one gradient
+ * per call.  The receive side (`dgc_decode_accumulate`, `dgc_apply_sgd`) is
+ * stateless.
+ *
+ * Conventions
+ *  - "device" pointers are CUDA device memory of the state's device, owned by
+ *    the caller unless stated; "host" pointers are ordinary host memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *    Calls that take a stream only enqueue work on it and return without
+ *    synchronising, unless stated.
+ *  - Every function returns DGC_OK (0) or a negative DGC_E* code; nothing
+ *    throws, aborts or prints.  dgc_error_string() names a code.
+ *  - There is no CPU fallback: without a usable CUDA device every call that
+ *    needs one returns DGC_ECUDA.
+ *
+ * Arena layout: tensor j occupies arena[arena_offset[j] .. + numel[j]); every
+ * tensor starts on a multiple of DGC_ARENA_ALIGN elements and the arena length
+ * is a multiple of it (dgc_layout reports the offsets).  The slots between
+ * tensors are padding: never selected, never written in u/v, decoded as +0.
+ * Their content in the gradient arena is ignored (it may be anything).
+ */
+#ifndef DGC_H_
+#define DGC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DGC_OK          0
+#define DGC_EINVAL     -1   /* bad argument                                   */
+#define DGC_ENOMEM     -2   /* device or host allocation failed               */
+#define DGC_ECAPACITY  -3   /* output buffer smaller than dgc_max_nnz()       */
+#define DGC_ECUDA      -4   /* a CUDA runtime call or kernel launch failed    */
+#define DGC_ESTATE     -5   /* state handle is NULL or already destroyed      */
+
+#define DGC_ARENA_ALIGN        512   /* elements; tensor starts and arena length */
+#define DGC_MAX_DECODE_WORKERS 64
+
+/* dgc_status.flags */
+#define DGC_FLAG_NONFINITE_NORM   1  /* the clipping norm was Inf or NaN            */
+#define DGC_FLAG_FULL_SELECT      2  /* a tensor needed the full-tensor selection   */
+#define DGC_FLAG_CAND_OVERFLOW    4  /* sampled threshold let too many entries pass */
+#define DGC_FLAG_CAND_SHORT       8  /* sampled threshold let fewer than k pass     */
+
+typedef struct dgc_state dgc_state;   /* opaque */
+
+typedef struct dgc_config {
+  int32_t        num_tensors;     /* M+1 of Algorithm 4; >= 1                                   */
+  int32_t        num_workers;     /* N: only enters the clip threshold thr_G * N^-1/2 (App. C)  */
+  const int64_t* tensor_numel;    /* host array [num_tensors], each >= 1; copied                */
+  float          momentum;        /* m of Eq. 5                                                 */
+  float          clip_threshold;  /* thr_G of Appendix C before the N^-1/2 scaling; <= 0: off   */
+  double         sparsity;        /* s in [0, 1): fraction of each tensor that is NOT sent      */
+  double         sample_ratio;    /* fraction of |v| sampled for the threshold estimate
+                                     (Sec. 5: 0.1% .. 1%); 0 selects the default 0.01           */
+  uint64_t       seed;            /* seed of the sampling positions                             */
+  int32_t        device;          /* CUDA device ordinal                                        */
+  int32_t        debug_sample_rank; /* test hook: when > 0, the sampled threshold is taken at
+                                     this rank of the sample instead of the safe one (rank 1 =
+                                     sample maximum, which forces the full-selection path)     */
+} dgc_config;
+
+typedef struct dgc_status {
+  double  grad_norm;          /* L2 norm of the last gradient set (0 when clipping is off)   */
+  float   clip_coef;          /* coefficient applied to the last gradient (1 = not clipped)  */
+  int32_t flags;              /* OR of DGC_FLAG_* over the last dgc_compress                 */
+  int64_t iterations;         /* dgc_compress calls so far                                   */
+  int64_t full_select_last;   /* tensors that took the full-selection path in the last call */
+  int64_t candidates_last;    /* entries that passed the sampled thresholds in the last call */
+} dgc_status;
+
+/* Algorithm 4, line "U^k <- 0, V^k <- 0": allocates and zeroes u and v (device
+ * memory of cfg->device, arena-sized), the selection scratch and the plan
+ * tables.  Synchronous.  The state is owned by the caller until
+ * dgc_state_destroy.  Errors: DGC_EINVAL (NULL, num_tensors < 1, numel < 1,
+ * sparsity outside [0,1), sample_ratio outside [0, 0.5], padded arena >=
+ * 2^31 elements), DGC_ENOMEM, DGC_ECUDA. */
+int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out);
+
+/* Frees everything dgc_state_create allocated.  Synchronises the device. */
+int32_t dgc_state_destroy(dgc_state* st);
+
+/* Sec. 3.3 "Warm-up Training" / Sec. 4.1: change the sparsity between two
+ * iterations.  Recomputes k_j = ceil(n_j (1 - s)) (integer arithmetic, parts
+ * per 1e9, at least 1), the output offsets and the sampling plan, and uploads
+ * them; may reallocate selection scratch (then it synchronises the device).
+ * Must not be called while a dgc_compress on this state is still running. */
+int32_t dgc_set_sparsity(dgc_state* st, double sparsity);
+
+/* Sec. 4.1: sparsity of warm-up stage 0..4 = 0.75, 0.9375, 0.984375, 0.996,
+ * 0.999.  DGC_EINVAL for other stages.  Host only. */
+int32_t dgc_warmup_sparsity(int32_t stage, double* sparsity_out);
+
+/* Sum over tensors of k_j: the exact number of pairs every dgc_compress call
+ * writes at the current sparsity.  Negative DGC_E* on error.  Host only. */
+int64_t dgc_max_nnz(const dgc_state* st);
+
+/* Host only.  Any output pointer may be NULL.
+ *   arena_offset[num_tensors]   first element of tensor j in the arena
+ *   k[num_tensors]              pairs emitted for tensor j per call
+ *   out_offset[num_tensors + 1] tensor j's pairs are out[out_offset[j] .. out_offset[j+1])
+ *   arena_len                   elements in the padded arena                          */
+int32_t dgc_layout(const dgc_state* st, int64_t* arena_offset, int64_t* k, int64_t* out_offset,
+                   int64_t* arena_len);
+
+/* One iteration of Algorithm 4 on this worker, from the clipping line to the
+ * end of the loop over tensors (Sec. 3.2, Eq. 5, Sec. 3.3, Sec. 5):
+ *   coef = min(1, thr_G N^-1/2 / ||g||_2) over the whole set (fp64 sum), gc = g*coef
+ *   u <- m*u + gc ; v <- v + u            (separately rounded fp32 operations)
+ *   per tensor j: the k_j entries of v largest in |v| (ties: lower index first)
+ *   out: their (arena index, v) pairs, ascending index, at out_offset[j]
+ *   v <- 0, u <- 0 at those entries (momentum factor masking)
+ * A seeded sample of |v| only proposes a threshold; the result is always the
+ * exact top-k_j set (if the proposal lets fewer than k_j or too many entries
+ * pass, that tensor is selected from the whole of v instead, see dgc_status).
+ *   grad_arena  device, const, arena_len floats, 16-byte aligned; not modified
+ *   out_idx     device, capacity int32   (index into the arena)
+ *   out_val     device, capacity floats
+ *   capacity    >= dgc_max_nnz(st), else DGC_ECAPACITY and nothing is enqueued
+ * Exactly dgc_max_nnz(st) pairs are written.  Asynchronous on `stream`; calls
+ * on one state must be stream-ordered with respect to each other, and the
+ * state's device must be the current device. */
+int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, float* out_val,
+                     int64_t capacity, void* stream);
+
+/* The same iteration with HOST buffers: copies grad_host (arena_len floats;
+ * pinned memory makes the copy asynchronous) into a staging buffer the state
+ * owns (allocated on first use), runs dgc_compress, copies the dgc_max_nnz(st)
+ * pairs back to out_idx_host / out_val_host and synchronises `stream`, so the
+ * lists are valid on return. */
+int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_idx_host,
+                          float* out_val_host, int64_t capacity, void* stream);
+
+/* Algorithm 4, line "G_t <- sum_k encode(G~_t^k)", for N workers' lists that
+ * already sit in this GPU's memory: dense_out[i] = (((+0 + val_0) + val_1) ...)
+ * over the workers that list index i, in worker order, fp32; +0 elsewhere.
+ * No floating-point atomics: each tile of dense_out is accumulated in shared
+ * memory one worker after the other and written once.
+ *   idx_lists, val_lists  host arrays [num_workers] of device pointers
+ *   nnz                   host array [num_workers], pairs per list (may be 0)
+ *   dense_out             device, dense_len floats, overwritten
+ *   workspace             device scratch of at least
+ *                         dgc_decode_workspace_bytes(num_workers, dense_len) bytes
+ * Precondition (not checked): each list's indices are strictly ascending and
+ * inside [0, dense_len) -- what dgc_compress produces.  1 <= num_workers <=
+ * DGC_MAX_DECODE_WORKERS.  Asynchronous on `stream`. */
+int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lists,
+                              const float* const* val_lists, const int64_t* nnz, float* dense_out,
+                              int64_t dense_len, void* workspace, int64_t workspace_bytes,
+                              void* stream);
+int64_t dgc_decode_workspace_bytes(int32_t num_workers, int64_t dense_len);
+
+/* Algorithm 4, line "theta <- SGD(theta, G_t)" with Eq. 5's third term:
+ * w[i] <- w[i] - lr * dense_grad[i], two separately rounded fp32 operations.
+ * w and dense_grad are device arrays of len floats.  Asynchronous. */
+int32_t dgc_apply_sgd(float* w, const float* dense_grad, int64_t len, float lr, void* stream);
+
+/* Synchronises `stream`, then reports counters of the last dgc_compress. */
+int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out);
+
+/* Synchronises `stream`, then copies per-tensor results of the last
+ * dgc_compress to host arrays [num_tensors] (either may be NULL):
+ *   kth_key     bit pattern of |v| of the smallest selected entry (the threshold of Algorithm 4)
+ *   candidates  entries that passed the sampled threshold (-1: full-selection path taken) */
+int32_t dgc_get_thresholds(dgc_state* st, void* stream, uint32_t* kth_key, int32_t* candidates);
+
+/* Checkpoint / resume: copy u and v (arena_len floats each) to / from host
+ * memory.  Synchronous on `stream`.  Either pointer may be NULL. */
+int32_t dgc_state_read(dgc_state* st, float* u_host, float* v_host, void* stream);
+int32_t dgc_state_write(dgc_state* st, const float* u_host, const float* v_host, void* stream);
+
+/* Number of kernels this library has launched in this process (all states). */
+uint64_t dgc_launch_count(void);
+
+const char* dgc_error_string(int32_t code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* DGC_H_ */

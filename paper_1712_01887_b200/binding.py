@@ -1,0 +1,227 @@
+"""Thin ctypes binding of the C ABI in include/dgc.h: argument marshalling only.
+
+Every step of the path runs in the CUDA library; there is no CPU fallback.
+Importing this module without the built library raises ImportError.
+PyTorch supplies device memory and streams: tensors are passed as raw device
+pointers, `stream` arguments default to torch's current stream.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libdgc.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_1712_01887_b200.build` "
+        "(there is no CPU fallback)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK, EINVAL, ENOMEM, ECAPACITY, ECUDA, ESTATE = 0, -1, -2, -3, -4, -5
+FLAG_NONFINITE_NORM, FLAG_FULL_SELECT, FLAG_CAND_OVERFLOW, FLAG_CAND_SHORT = 1, 2, 4, 8
+ARENA_ALIGN = 512
+MAX_DECODE_WORKERS = 64
+
+
+class Config(ctypes.Structure):
+    _fields_ = [("num_tensors", ctypes.c_int32), ("num_workers", ctypes.c_int32),
+                ("tensor_numel", ctypes.POINTER(ctypes.c_int64)), ("momentum", ctypes.c_float),
+                ("clip_threshold", ctypes.c_float), ("sparsity", ctypes.c_double),
+                ("sample_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
+                ("device", ctypes.c_int32), ("debug_sample_rank", ctypes.c_int32)]
+
+
+class Status(ctypes.Structure):
+    _fields_ = [("grad_norm", ctypes.c_double), ("clip_coef", ctypes.c_float),
+                ("flags", ctypes.c_int32), ("iterations", ctypes.c_int64),
+                ("full_select_last", ctypes.c_int64), ("candidates_last", ctypes.c_int64)]
+
+
+_vp = ctypes.c_void_p
+_i64p = ctypes.POINTER(ctypes.c_int64)
+_sigs = {
+    "dgc_state_create": (ctypes.c_int32, [ctypes.POINTER(Config), ctypes.POINTER(_vp)]),
+    "dgc_state_destroy": (ctypes.c_int32, [_vp]),
+    "dgc_set_sparsity": (ctypes.c_int32, [_vp, ctypes.c_double]),
+    "dgc_warmup_sparsity": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(ctypes.c_double)]),
+    "dgc_max_nnz": (ctypes.c_int64, [_vp]),
+    "dgc_layout": (ctypes.c_int32, [_vp, _i64p, _i64p, _i64p, _i64p]),
+    "dgc_compress": (ctypes.c_int32, [_vp, _vp, _vp, _vp, ctypes.c_int64, _vp]),
+    "dgc_compress_host": (ctypes.c_int32, [_vp, _vp, _vp, _vp, ctypes.c_int64, _vp]),
+    "dgc_decode_accumulate": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
+                                               ctypes.POINTER(_vp), _i64p, _vp, ctypes.c_int64,
+                                               _vp, ctypes.c_int64, _vp]),
+    "dgc_decode_workspace_bytes": (ctypes.c_int64, [ctypes.c_int32, ctypes.c_int64]),
+    "dgc_apply_sgd": (ctypes.c_int32, [_vp, _vp, ctypes.c_int64, ctypes.c_float, _vp]),
+    "dgc_get_status": (ctypes.c_int32, [_vp, _vp, ctypes.POINTER(Status)]),
+    "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
+    "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
+    "dgc_state_write": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
+    "dgc_launch_count": (ctypes.c_uint64, []),
+    "dgc_error_string": (ctypes.c_char_p, [ctypes.c_int32]),
+}
+for _name, (_res, _args) in _sigs.items():
+    _fn = getattr(_lib, _name)
+    _fn.restype = _res
+    _fn.argtypes = _args
+
+EXPORTED = tuple(_sigs)
+
+
+class DgcError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        super().__init__(f"{where}: {_lib.dgc_error_string(int(code)).decode()} ({code})")
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise DgcError(code, where)
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, torch.cuda.Stream):
+        return stream.cuda_stream
+    return int(stream)
+
+
+def _dev(t: torch.Tensor, dtype) -> int:
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise ValueError(f"expected a contiguous CUDA {dtype} tensor")
+    return t.data_ptr()
+
+
+def warmup_sparsity(stage: int) -> float:
+    s = ctypes.c_double()
+    _check(_lib.dgc_warmup_sparsity(int(stage), ctypes.byref(s)), "dgc_warmup_sparsity")
+    return s.value
+
+
+def launch_count() -> int:
+    return int(_lib.dgc_launch_count())
+
+
+class State:
+    """One worker of Algorithm 4: owns u and v on the device."""
+
+    def __init__(self, tensor_numel: Sequence[int], num_workers: int, momentum: float,
+                 clip_threshold: float, sparsity: float, sample_ratio: float = 0.01,
+                 seed: int = 0, device: int = 0, debug_sample_rank: int = 0):
+        numel = (ctypes.c_int64 * len(tensor_numel))(*[int(n) for n in tensor_numel])
+        cfg = Config(len(tensor_numel), int(num_workers), numel, float(momentum),
+                     float(clip_threshold), float(sparsity), float(sample_ratio), int(seed),
+                     int(device), int(debug_sample_rank))
+        self._h = _vp()
+        self.num_tensors = len(tensor_numel)
+        self.device = int(device)
+        _check(_lib.dgc_state_create(ctypes.byref(cfg), ctypes.byref(self._h)), "dgc_state_create")
+        self._refresh_layout()
+
+    def _refresh_layout(self) -> None:
+        T = self.num_tensors
+        off = np.zeros(T, np.int64)
+        k = np.zeros(T, np.int64)
+        out = np.zeros(T + 1, np.int64)
+        alen = ctypes.c_int64()
+        _check(_lib.dgc_layout(self._h, off.ctypes.data_as(_i64p), k.ctypes.data_as(_i64p),
+                               out.ctypes.data_as(_i64p), ctypes.byref(alen)), "dgc_layout")
+        self.arena_offset, self.k, self.out_offset, self.arena_len = off, k, out, int(alen.value)
+        self.max_nnz = int(_lib.dgc_max_nnz(self._h))
+
+    def close(self) -> None:
+        if self._h:
+            _check(_lib.dgc_state_destroy(self._h), "dgc_state_destroy")
+            self._h = _vp()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def set_sparsity(self, sparsity: float) -> None:
+        _check(_lib.dgc_set_sparsity(self._h, float(sparsity)), "dgc_set_sparsity")
+        self._refresh_layout()
+
+    def compress(self, grad: torch.Tensor, out_idx: torch.Tensor, out_val: torch.Tensor,
+                 stream=None) -> None:
+        if grad.numel() != self.arena_len:
+            raise ValueError("gradient arena has the wrong length")
+        cap = min(out_idx.numel(), out_val.numel())
+        _check(_lib.dgc_compress(self._h, _dev(grad, torch.float32), _dev(out_idx, torch.int32),
+                                 _dev(out_val, torch.float32), cap, _stream(stream)),
+               "dgc_compress")
+
+    def compress_host(self, grad: torch.Tensor, out_idx: torch.Tensor, out_val: torch.Tensor,
+                      stream=None) -> None:
+        for t, dt in ((grad, torch.float32), (out_idx, torch.int32), (out_val, torch.float32)):
+            if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+                raise ValueError("expected contiguous host tensors")
+        if grad.numel() != self.arena_len:
+            raise ValueError("gradient arena has the wrong length")
+        cap = min(out_idx.numel(), out_val.numel())
+        _check(_lib.dgc_compress_host(self._h, grad.data_ptr(), out_idx.data_ptr(),
+                                      out_val.data_ptr(), cap, _stream(stream)),
+               "dgc_compress_host")
+
+    def status(self, stream=None) -> Status:
+        s = Status()
+        _check(_lib.dgc_get_status(self._h, _stream(stream), ctypes.byref(s)), "dgc_get_status")
+        return s
+
+    def thresholds(self, stream=None):
+        kth = np.zeros(self.num_tensors, np.uint32)
+        cand = np.zeros(self.num_tensors, np.int32)
+        _check(_lib.dgc_get_thresholds(self._h, _stream(stream), kth.ctypes.data, cand.ctypes.data),
+               "dgc_get_thresholds")
+        return kth, cand
+
+    def read(self, stream=None):
+        u = np.empty(self.arena_len, np.float32)
+        v = np.empty(self.arena_len, np.float32)
+        _check(_lib.dgc_state_read(self._h, u.ctypes.data, v.ctypes.data, _stream(stream)),
+               "dgc_state_read")
+        return u, v
+
+    def write(self, u: Optional[np.ndarray], v: Optional[np.ndarray], stream=None) -> None:
+        for a in (u, v):
+            if a is not None and (a.dtype != np.float32 or a.size != self.arena_len
+                                  or not a.flags["C_CONTIGUOUS"]):
+                raise ValueError("expected contiguous float32 arrays of arena_len")
+        _check(_lib.dgc_state_write(self._h, None if u is None else u.ctypes.data,
+                                    None if v is None else v.ctypes.data, _stream(stream)),
+               "dgc_state_write")
+
+
+def decode_workspace_bytes(num_workers: int, dense_len: int) -> int:
+    return int(_lib.dgc_decode_workspace_bytes(int(num_workers), int(dense_len)))
+
+
+def decode_accumulate(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[torch.Tensor],
+                      dense_out: torch.Tensor, workspace: torch.Tensor, stream=None,
+                      nnz: Optional[Sequence[int]] = None) -> None:
+    n = len(idx_lists)
+    ip = (_vp * n)(*[_dev(t, torch.int32) for t in idx_lists])
+    vp = (_vp * n)(*[_dev(t, torch.float32) for t in val_lists])
+    cnt = (ctypes.c_int64 * n)(*[int(c) for c in (nnz if nnz is not None
+                                                  else [t.numel() for t in idx_lists])])
+    _check(_lib.dgc_decode_accumulate(n, ip, vp, cnt, _dev(dense_out, torch.float32),
+                                      dense_out.numel(), workspace.data_ptr(),
+                                      workspace.numel() * workspace.element_size(),
+                                      _stream(stream)), "dgc_decode_accumulate")
+
+
+def apply_sgd(w: torch.Tensor, dense_grad: torch.Tensor, lr: float, stream=None) -> None:
+    if w.numel() != dense_grad.numel():
+        raise ValueError("length mismatch")
+    _check(_lib.dgc_apply_sgd(_dev(w, torch.float32), _dev(dense_grad, torch.float32), w.numel(),
+                              float(lr), _stream(stream)), "dgc_apply_sgd")

@@ -1,0 +1,282 @@
+"""GPU parity: the CUDA library (called through the C ABI) against the CPU
+oracle on the same seeded inputs.  Bit-exact for indices, sent values, u, v,
+decoded sums and weights; clipping norm within 1e-6 relative."""
+import numpy as np
+import pytest
+import torch
+
+from paper_1712_01887_b200 import inputs as I
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    if not torch.cuda.is_available():
+        pytest.fail("no CUDA device: the gpu tests need a B200")
+    import parity_util
+    return parity_util
+
+
+def _run_workload(P, wl, iterations, workers=None, seed=0, receive=True, schedule=None,
+                  check_state=True):
+    N = workers or wl.num_workers
+    pairs = [P.Pair(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold, wl.sparsity,
+                    seed=seed + w, sample_ratio=wl.sample_ratio) for w in range(N)]
+    rep = P.ParityReport()
+    off, L = pairs[0].gpu.arena_offset, pairs[0].gpu.arena_len
+    rng = np.random.default_rng(99)
+    w_host = rng.standard_normal(L).astype(np.float32)
+    for t in range(iterations):
+        if schedule is not None:
+            s = schedule(t)
+            if s != pairs[0].cpu.sparsity:
+                for p in pairs:
+                    p.set_sparsity(s)
+        lists_i, lists_v = [], []
+        for w, p in enumerate(pairs):
+            g = P.arena_with_padding_poison(L, off, wl.numel)
+            I.fill(wl, g, off, worker=w, iteration=t)
+            gi, gv, _ = p.step(g, rep, check_state=check_state)
+            lists_i.append(gi)
+            lists_v.append(gv)
+        if receive:
+            _, w_host = P.receive_side(lists_i, lists_v, L, w_host, lr=0.1)
+    for p in pairs:
+        p.close()
+    assert rep.near_threshold_ties == 0
+    return rep
+
+
+def test_cfg1_outlier_tensor_5_iterations(P):
+    wl = I.workload("cfg1")
+    rep = _run_workload(P, wl, wl.iterations)
+    assert rep.worker_iterations == 20
+    assert rep.full_select == 0
+
+
+def test_resnet50_shapes_two_workers(P):
+    wl = I.workload("resnet50")
+    rep = _run_workload(P, wl, 3, workers=2)
+    assert rep.full_select == 0
+
+
+def test_resnet50_shapes_with_clipping(P):
+    wl = I.workload("resnet50")
+    wl.clip_threshold = 1.0
+    _run_workload(P, wl, 2, workers=1, receive=False)
+
+
+def test_lstm_small_row_sparse_embedding(P):
+    wl = I.workload("lstm_small")
+    _run_workload(P, wl, 4)
+
+
+def test_deepspeech_small_warmup_schedule(P):
+    wl = I.workload("deepspeech_small")
+    stages = [0.75, 0.9375, 0.984375, 0.996, 0.999]
+    _run_workload(P, wl, 10, workers=2, schedule=lambda t: stages[min(t // 2, 4)])
+
+
+@pytest.mark.parametrize("sparsity", [0.999, 0.99, 0.75, 0.0])
+def test_edge_sizes(P, sparsity):
+    numel = [1, 3, 4, 5, 31, 32, 33, 511, 512, 513, 4095, 4096, 4097, 8192, 8193, 70001,
+             524288, 524289]
+    wl = I.Workload("edge", [(n,) for n in numel], 4, 0.9, 1.0, sparsity, 3, "normal")
+    _run_workload(P, wl, 3, workers=1)
+
+
+def test_heavy_ties_and_zeros(P):
+    """Quantised values: thousands of exact ties at the threshold; ties go to the lower index."""
+    numel = [100000, 5000, 300000]
+    pair = P.Pair(numel, 2, 0.5, 0.0, 0.99, seed=3)
+    rep = P.ParityReport()
+    rng = np.random.default_rng(5)
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    for t in range(4):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for o, n in zip(off, numel):
+            g[o:o + n] = rng.integers(-3, 4, size=n).astype(np.float32) * np.float32(0.25)
+        pair.step(g, rep)
+    pair.close()
+
+
+def test_all_zero_gradient_takes_full_selection_and_picks_lowest_indices(P):
+    numel = [20000, 100]
+    pair = P.Pair(numel, 1, 0.9, 0.0, 0.999, seed=1)
+    rep = P.ParityReport()
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    g = P.arena_with_padding_poison(L, off, numel)
+    gi, gv, st = pair.step(g, rep)
+    assert gi.tolist() == list(range(20)) + [int(off[1])]
+    assert not gv.any()
+    assert st.flags & 2 and st.full_select_last >= 1
+    pair.close()
+
+
+def test_forced_full_selection_path_matches(P):
+    """debug_sample_rank = 1 proposes the sample maximum: too few pass, every sampled tensor
+    falls back to selecting from the whole of v; the result must not change."""
+    numel = [50000, 9000, 1200000, 64]
+    pair = P.Pair(numel, 1, 0.9, 0.0, 0.999, seed=2, debug_sample_rank=1)
+    rep = P.ParityReport()
+    rng = np.random.default_rng(8)
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    for t in range(3):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for o, n in zip(off, numel):
+            g[o:o + n] = rng.standard_normal(n).astype(np.float32)
+        _, _, st = pair.step(g, rep)
+        # the 9000-entry tensor may still get k candidates above its sample maximum
+        assert st.full_select_last >= 2 and st.flags & 8
+    pair.close()
+
+
+def test_result_independent_of_sampling_seed_and_ratio(P):
+    numel = [300000, 40000]
+    rng = np.random.default_rng(12)
+    grads = []
+    outs = []
+    for seed, ratio in ((1, 0.01), (2, 0.001), (3, 0.005)):
+        pair = P.Pair(numel, 1, 0.9, 0.0, 0.999, seed=seed, sample_ratio=ratio)
+        off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+        if not grads:
+            for t in range(3):
+                g = P.arena_with_padding_poison(L, off, numel)
+                for o, n in zip(off, numel):
+                    g[o:o + n] = rng.standard_t(3, n).astype(np.float32)
+                grads.append(g)
+        rep = P.ParityReport()
+        res = [pair.step(g, rep)[0].copy() for g in grads]
+        outs.append(res)
+        pair.close()
+    for other in outs[1:]:
+        for a, b in zip(outs[0], other):
+            assert np.array_equal(a, b)
+
+
+def test_special_values_inf_and_nan_are_selected_first(P):
+    numel = [10000]
+    pair = P.Pair(numel, 1, 0.9, 0.0, 0.999, seed=4)     # k = 10
+    rep = P.ParityReport()
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    rng = np.random.default_rng(1)
+    g = P.arena_with_padding_poison(L, off, numel)
+    g[:10000] = rng.standard_normal(10000).astype(np.float32)
+    g[5000] = np.inf
+    g[5001] = -np.inf
+    gi, gv, _ = pair.step(g, rep)
+    assert {5000, 5001} <= set(gi.tolist())
+    # NaN: its payload may differ between CPU and GPU arithmetic, so only the GPU's choice
+    # is checked here: the NaN entry has the largest key and is sent
+    g[:10000] = rng.standard_normal(10000).astype(np.float32)
+    g[77] = np.nan
+    pair.gpu.compress(torch.from_numpy(g).cuda(), pair.out_idx, pair.out_val)
+    sel = pair.out_idx.cpu().numpy()
+    assert 77 in sel.tolist() and np.isnan(pair.out_val.cpu().numpy()[sel.tolist().index(77)])
+    pair.close()
+
+
+def test_deterministic_across_runs(P):
+    wl = I.workload("sweep", n=1 << 21)
+    outs = []
+    for _ in range(2):
+        pair = P.Pair(wl.numel, 1, 0.9, 0.5, 0.999, seed=9)
+        off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+        res = []
+        for t in range(3):
+            g = np.zeros(L, np.float32)
+            I.fill(wl, g, off, 0, t)
+            gd = torch.from_numpy(g).cuda()
+            pair.gpu.compress(gd, pair.out_idx, pair.out_val)
+            u, v = pair.gpu.read()
+            res.append((pair.out_idx.cpu().numpy().copy(), pair.out_val.cpu().numpy().copy(), u, v,
+                        pair.gpu.status().grad_norm))
+        outs.append(res)
+        pair.close()
+    for a, b in zip(*outs):
+        for x, y in zip(a[:4], b[:4]):
+            assert x.tobytes() == y.tobytes()
+        assert a[4] == b[4]
+
+
+def test_checkpoint_resume_is_bit_identical(P):
+    from paper_1712_01887_b200 import binding as B
+    numel = [100000, 777]
+    rng = np.random.default_rng(3)
+    a = B.State(numel, 1, 0.9, 0.0, 0.999, seed=5)
+    L = a.arena_len
+    gs = [torch.from_numpy(rng.standard_normal(L).astype(np.float32)).cuda() for _ in range(3)]
+    oi = torch.empty(a.max_nnz, dtype=torch.int32, device="cuda")
+    ov = torch.empty(a.max_nnz, dtype=torch.float32, device="cuda")
+    a.compress(gs[0], oi, ov)
+    a.compress(gs[1], oi, ov)
+    u, v = a.read()
+    b = B.State(numel, 1, 0.9, 0.0, 0.999, seed=5)
+    b.write(u, v)
+    a.compress(gs[2], oi, ov)
+    oi2, ov2 = torch.empty_like(oi), torch.empty_like(ov)
+    b.compress(gs[2], oi2, ov2)
+    assert torch.equal(oi, oi2) and torch.equal(ov.view(torch.int32), ov2.view(torch.int32))
+    ua, va = a.read()
+    ub, vb = b.read()
+    assert ua.tobytes() == ub.tobytes() and va.tobytes() == vb.tobytes()
+    a.close()
+    b.close()
+
+
+def test_compress_host_matches_device_path(P):
+    from paper_1712_01887_b200 import binding as B
+    numel = [200000, 3000]
+    rng = np.random.default_rng(6)
+    a = B.State(numel, 4, 0.9, 1.0, 0.999, seed=5)
+    b = B.State(numel, 4, 0.9, 1.0, 0.999, seed=5)
+    L = a.arena_len
+    for t in range(2):
+        gh = torch.from_numpy(rng.standard_normal(L).astype(np.float32)).pin_memory()
+        oi = torch.empty(a.max_nnz, dtype=torch.int32, device="cuda")
+        ov = torch.empty(a.max_nnz, dtype=torch.float32, device="cuda")
+        a.compress(gh.cuda(), oi, ov)
+        hi = torch.empty(a.max_nnz, dtype=torch.int32).pin_memory()
+        hv = torch.empty(a.max_nnz, dtype=torch.float32).pin_memory()
+        b.compress_host(gh, hi, hv)
+        assert torch.equal(oi.cpu(), hi) and torch.equal(ov.cpu().view(torch.int32), hv.view(torch.int32))
+    a.close()
+    b.close()
+
+
+def test_abi_errors(P):
+    from paper_1712_01887_b200 import binding as B
+    with pytest.raises(B.DgcError) as e:
+        B.State([0], 1, 0.9, 0.0, 0.999)
+    assert e.value.code == B.EINVAL
+    with pytest.raises(B.DgcError):
+        B.State([10], 1, 0.9, 0.0, 1.0)
+    st = B.State([5000], 1, 0.9, 0.0, 0.99)
+    g = torch.zeros(st.arena_len, device="cuda")
+    small_i = torch.empty(st.max_nnz - 1, dtype=torch.int32, device="cuda")
+    small_v = torch.empty(st.max_nnz - 1, dtype=torch.float32, device="cuda")
+    with pytest.raises(B.DgcError) as e:
+        st.compress(g, small_i, small_v)
+    assert e.value.code == B.ECAPACITY
+    with pytest.raises(B.DgcError) as e:
+        st.set_sparsity(1.5)
+    assert e.value.code == B.EINVAL
+    st.close()
+    with pytest.raises(B.DgcError) as e:
+        st.set_sparsity(0.5)
+    assert e.value.code == B.ESTATE
+
+
+def test_decode_edge_cases(P):
+    rng = np.random.default_rng(17)
+    for L, N, density in ((1, 1, 1.0), (4095, 3, 0.01), (4096, 2, 0.5), (4097, 5, 0.001),
+                          (1 << 20, 8, 0.001), (100003, 64, 0.01), (50000, 4, 1.0), (9000, 2, 0.0)):
+        idx, val = [], []
+        for w in range(N):
+            k = int(round(L * density)) if w % 2 == 0 else int(L * density / 2)
+            i = np.sort(rng.choice(L, size=min(k, L), replace=False)).astype(np.int32)
+            idx.append(i)
+            val.append(rng.standard_normal(i.size).astype(np.float32))
+        w0 = rng.standard_normal(L).astype(np.float32)
+        P.receive_side(idx, val, L, w0, lr=0.05)
