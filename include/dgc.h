@@ -176,6 +176,15 @@ int32_t dgc_get_thresholds(dgc_state* st, void* stream, uint32_t* kth_key, int32
 int32_t dgc_state_read(dgc_state* st, float* u_host, float* v_host, void* stream);
 int32_t dgc_state_write(dgc_state* st, const float* u_host, const float* v_host, void* stream);
 
+/* Measurement aid (not part of the method): after dgc_profile_enable(st, n) the
+ * next n dgc_compress calls record a CUDA event pair around their streaming
+ * kernel (the fused Eq. 5 update + candidate emission pass) on the call's
+ * stream.  dgc_profile_read waits for the recorded pairs and returns their
+ * durations in milliseconds (ms_out[capacity], *count_out = pairs returned).
+ * dgc_profile_enable(st, 0) switches recording off. */
+int32_t dgc_profile_enable(dgc_state* st, int32_t max_calls);
+int32_t dgc_profile_read(dgc_state* st, float* ms_out, int32_t capacity, int32_t* count_out);
+
 /* Number of kernels this library has launched in this process (all states). */
 uint64_t dgc_launch_count(void);
 

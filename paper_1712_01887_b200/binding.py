@@ -64,6 +64,9 @@ _sigs = {
     "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_write": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
+    "dgc_profile_enable": (ctypes.c_int32, [_vp, ctypes.c_int32]),
+    "dgc_profile_read": (ctypes.c_int32, [_vp, _vp, ctypes.c_int32,
+                                          ctypes.POINTER(ctypes.c_int32)]),
     "dgc_launch_count": (ctypes.c_uint64, []),
     "dgc_error_string": (ctypes.c_char_p, [ctypes.c_int32]),
 }
@@ -184,6 +187,16 @@ class State:
         _check(_lib.dgc_get_thresholds(self._h, _stream(stream), kth.ctypes.data, cand.ctypes.data),
                "dgc_get_thresholds")
         return kth, cand
+
+    def profile_enable(self, max_calls: int) -> None:
+        _check(_lib.dgc_profile_enable(self._h, int(max_calls)), "dgc_profile_enable")
+
+    def profile_read(self, capacity: int) -> np.ndarray:
+        ms = np.zeros(max(int(capacity), 1), np.float32)
+        n = ctypes.c_int32()
+        _check(_lib.dgc_profile_read(self._h, ms.ctypes.data, int(capacity), ctypes.byref(n)),
+               "dgc_profile_read")
+        return ms[:n.value].copy()
 
     def read(self, stream=None):
         u = np.empty(self.arena_len, np.float32)

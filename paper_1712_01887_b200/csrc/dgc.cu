@@ -37,13 +37,15 @@ namespace {
 
 // ------------------------------------------------------------------ constants
 constexpr int kSeg = 512;              // elements per warp segment (4 x float4 per lane)
-constexpr int kPartSegs = 1024;        // segments per part (512 Ki elements)
+constexpr int kPartSegs = 512;         // segments per part (256 Ki elements)
 constexpr int kSmallN = 8192;          // tensors up to this size are not sampled
 constexpr int kMaxSampleGroups = 3072; // float4 groups sampled per tensor at most
 constexpr int kSampleThreads = 512;
 constexpr int kSelectThreads = 1024;
 constexpr int kSelectMaxSmemKeys = 49152;
-constexpr int kEmitThreads = 512;
+constexpr int kEmitThreads = kPartSegs;   // one thread per segment of the part
+constexpr int kMaskStride = 17;           // words per segment in the winner bitmaps (16 + 1 pad)
+constexpr int kEmitSmemBytes = 2 * kPartSegs * kMaskStride * 4;
 constexpr int kMainThreads = 256;
 constexpr int kNormThreads = 256;
 constexpr int kMaxNormGrid = 2048;
@@ -164,10 +166,19 @@ __device__ uint32_t block_select_desc(ForEach for_each, int rank, uint32_t* hist
     for (int i = tid; i < 256; i += nt) hist[i] = 0;
     __syncthreads();
     for_each([&](bool valid, uint32_t key) {
-      uint32_t d = 0x100u + lane;             // unique per lane: never aggregated, never added
+      uint32_t d = 0;
       if (valid && (key & mask) == prefix) d = (key >> shift) & 255u; else valid = false;
-      const unsigned peers = __match_any_sync(0xFFFFFFFFu, d);
-      if (valid && lane == __ffs(peers) - 1) atomicAdd(&hist[d], (uint32_t)__popc(peers));
+      // keys cluster on a few digits in the leading passes: lanes that share the digit of
+      // the first valid lane are added with one atomic, the others one by one
+      const unsigned vm = __ballot_sync(0xFFFFFFFFu, valid);
+      if (vm != 0) {
+        const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, d, __ffs(vm) - 1);
+        const unsigned m0 = __ballot_sync(0xFFFFFFFFu, valid && d == d0);
+        if (valid) {
+          if (d != d0) atomicAdd(&hist[d], 1u);
+          else if (lane == __ffs(m0) - 1) atomicAdd(&hist[d], (uint32_t)__popc(m0));
+        }
+      }
     });
     __syncthreads();
     if (tid < 32) {
@@ -588,11 +599,12 @@ k_select(Plan p, int smem_keys, int parity) {
 
 // ------------------------------------------------------------------ K5: ordered emission + masking
 // Algorithm 4: G~[j] <- V[j] (.) Mask ; V[j] <- V[j] (.) !Mask ; U[j] <- U[j] (.) !Mask.
-// One block per part.  A part's candidate list is a sequence of runs, one run
-// per segment, each run ascending in index; the number of winners in earlier
-// segments comes from per-segment counts (shared-memory integer atomics) and an
-// exclusive scan, the number of earlier winners inside the run from walking the
-// run backwards.
+// One block per part, one thread per segment.  The candidates that reach the
+// threshold set one bit each in a shared-memory bitmap of the part (integer
+// atomicOr; "greater" and "tied" bitmaps); per-segment popcounts and an
+// exclusive scan give every segment its first output slot; each thread then
+// walks its segment's bits in index order, reads v' at those entries, writes
+// the pairs and zeroes u and v there.
 //
 // Full-selection path (dense flag set by k_select): the block of the tensor's
 // first part selects from the whole of v' (radix select over global memory) and
@@ -656,10 +668,11 @@ __device__ void dense_select_emit(const Plan& p, int j, int32_t* out_idx, float*
 
 __global__ void __launch_bounds__(kEmitThreads)
 k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
-  __shared__ int s_gt[kPartSegs];
-  __shared__ int s_eq[kPartSegs];
+  extern __shared__ uint32_t smask[];          // winner bitmaps of the part: [gt | eq]
   __shared__ uint32_t hist[256];
   __shared__ int sh[40];
+  uint32_t* mgt = smask;
+  uint32_t* meq = smask + kPartSegs * kMaskStride;
   const int part = blockIdx.x;
   const int tid = threadIdx.x;
   const int j = p.p_tensor[part];
@@ -678,64 +691,50 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   const int nseg = p.p_nseg[part];
   const int32_t* cidx = p.cand_idx + p.p_cbase[part];
   const float* cval = p.cand_val + p.p_cbase[part];
-  for (int s = tid; s < nseg; s += kEmitThreads) { s_gt[s] = 0; s_eq[s] = 0; }
+  for (int i = tid; i < 2 * kPartSegs * kMaskStride; i += kEmitThreads) smask[i] = 0u;
   __syncthreads();
+  // mark the candidates that reach the threshold: one bit per element of the part
   for (int i = tid; i < count; i += kEmitThreads) {
     const uint32_t key = mag_key(__ldcg(cval + i));
     if (key >= kth) {
-      const int s = (__ldcg(cidx + i) >> 9) - seg0;
-      if (key > kth) atomicAdd(&s_gt[s], 1); else atomicAdd(&s_eq[s], 1);
+      const int local = __ldcg(cidx + i) - seg0 * kSeg;
+      const int word = (local >> 9) * kMaskStride + ((local >> 5) & 15);
+      atomicOr((key > kth ? mgt : meq) + word, 1u << (local & 31));
     }
   }
   __syncthreads();
-  // exclusive scan over the part's segments, in place (2 segments per thread)
-  {
-    constexpr int kPer = kPartSegs / kEmitThreads;
-    int g[kPer], e[kPer], sg = 0, se = 0;
+  // thread s owns segment s: count, scan, then walk its bits in index order
+  int gt = 0, eq = 0;
+  if (tid < nseg) {
 #pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-      const int s = tid * kPer + q;
-      g[q] = s < nseg ? s_gt[s] : 0;
-      e[q] = s < nseg ? s_eq[s] : 0;
-      sg += g[q];
-      se += e[q];
-    }
-    int tg, te;
-    int bg = block_excl_scan(sg, sh, tg);
-    int be = block_excl_scan(se, sh, te);
-#pragma unroll
-    for (int q = 0; q < kPer; ++q) {
-      const int s = tid * kPer + q;
-      if (s < nseg) { s_gt[s] = bg; s_eq[s] = be; }
-      bg += g[q];
-      be += e[q];
+    for (int w = 0; w < 16; ++w) {
+      gt += __popc(mgt[tid * kMaskStride + w]);
+      eq += __popc(meq[tid * kMaskStride + w]);
     }
   }
-  __syncthreads();
-  for (int i = tid; i < count; i += kEmitThreads) {
-    const float val = __ldcg(cval + i);
-    const uint32_t key = mag_key(val);
-    if (key < kth) continue;
-    const int idx = __ldcg(cidx + i);
-    const int sabs = idx >> 9;
-    // winners earlier in this segment's run
-    int lg = 0, le = 0;
-    for (int b = i - 1; b >= 0; --b) {
-      if ((__ldcg(cidx + b) >> 9) != sabs) break;
-      const uint32_t kb = mag_key(__ldcg(cval + b));
-      lg += kb > kth;
-      le += kb == kth;
-    }
-    const int s = sabs - seg0;
-    const int eq_before = s_eq[s];
-    const int left = max(0, quota - eq_before);        // ties this segment may still take
-    const bool take = key > kth || le < left;
-    if (take) {
-      const int pos = out_base + s_gt[s] + min(eq_before, quota) + lg + min(le, left);
-      out_idx[pos] = idx;
-      out_val[pos] = val;
-      p.u[idx] = 0.0f;
-      p.v[idx] = 0.0f;
+  int tg, te;
+  const int bg = block_excl_scan(gt, sh, tg);
+  int eqr = block_excl_scan(eq, sh, te);
+  if (gt + eq == 0) return;
+  int pos = out_base + bg + min(eqr, quota);
+  const int ebase = (seg0 + tid) * kSeg;
+  for (int w = 0; w < 16; ++w) {
+    const uint32_t g = mgt[tid * kMaskStride + w];
+    const uint32_t e = meq[tid * kMaskStride + w];
+    uint32_t both = g | e;
+    while (both) {
+      const int b = __ffs(both) - 1;
+      both &= both - 1;
+      bool take = true;
+      if ((e >> b) & 1u) { take = eqr < quota; ++eqr; }   // ties: lowest indices first
+      if (take) {
+        const int idx = ebase + w * 32 + b;
+        out_idx[pos] = idx;
+        out_val[pos] = __ldcg(p.v + idx);
+        p.u[idx] = 0.0f;
+        p.v[idx] = 0.0f;
+        ++pos;
+      }
     }
   }
 }
@@ -886,6 +885,9 @@ struct dgc_state {
   float* d_stage_val = nullptr;
   int64_t stage_nnz = 0;
   Plan plan{};
+  // optional timing of the streaming kernel (dgc_profile_enable)
+  std::vector<cudaEvent_t> prof_ev;   // 2 events per recorded call
+  int prof_cap = 0, prof_n = 0;
   int norm_grid = 0, main_grid = 0, main_grid_clip = 0;
   int select_smem_keys = 0;
   bool alive = false;
@@ -1161,6 +1163,8 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
                            kMaxSampleGroups * 16) != cudaSuccess) return fail(DGC_ECUDA);
   if (cudaFuncSetAttribute(k_sample_threshold<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kMaxSampleGroups * 16) != cudaSuccess) return fail(DGC_ECUDA);
+  if (cudaFuncSetAttribute(k_emit_mask, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           kEmitSmemBytes) != cudaSuccess) return fail(DGC_ECUDA);
   if (cudaDeviceSynchronize() != cudaSuccess) return fail(DGC_ECUDA);
   *out = st;
   return DGC_OK;
@@ -1172,6 +1176,8 @@ int32_t dgc_state_destroy(dgc_state* st) {
   cudaDeviceSynchronize();
   for (void* ptr : st->allocs) cudaFree(ptr);
   st->allocs.clear();
+  for (cudaEvent_t e : st->prof_ev) cudaEventDestroy(e);
+  st->prof_ev.clear();
   st->alive = false;
   delete st;
   return DGC_OK;
@@ -1232,15 +1238,21 @@ int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, f
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   {
+    const bool prof = st->prof_n < st->prof_cap;
+    if (prof) DGC_CUDA(cudaEventRecord(st->prof_ev[2 * st->prof_n], s));
     const int need = (p.num_segs + (kMainThreads / 32) - 1) / (kMainThreads / 32);
     if (clip) k_update_emit<true><<<std::min(st->main_grid_clip, need), kMainThreads, 0, s>>>(p, grad_arena, m);
     else k_update_emit<false><<<std::min(st->main_grid, need), kMainThreads, 0, s>>>(p, grad_arena, m);
     if ((rc = check_launch()) != DGC_OK) return rc;
+    if (prof) {
+      DGC_CUDA(cudaEventRecord(st->prof_ev[2 * st->prof_n + 1], s));
+      st->prof_n += 1;
+    }
   }
   k_select<<<p.num_tensors, kSelectThreads, (size_t)st->select_smem_keys * 4, s>>>(
       p, st->select_smem_keys, parity);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_emit_mask<<<p.num_parts, kEmitThreads, 0, s>>>(p, out_idx, out_val);
+  k_emit_mask<<<p.num_parts, kEmitThreads, kEmitSmemBytes, s>>>(p, out_idx, out_val);
   if ((rc = check_launch()) != DGC_OK) return rc;
   st->iterations += 1;
   return DGC_OK;
@@ -1360,6 +1372,32 @@ int32_t dgc_get_thresholds(dgc_state* st, void* stream, uint32_t* kth_key, int32
   const size_t T = st->cfg.num_tensors;
   if (kth_key) DGC_CUDA(cudaMemcpy(kth_key, st->plan.t_kth, T * 4, cudaMemcpyDeviceToHost));
   if (candidates) DGC_CUDA(cudaMemcpy(candidates, st->plan.t_cand, T * 4, cudaMemcpyDeviceToHost));
+  return DGC_OK;
+}
+
+int32_t dgc_profile_enable(dgc_state* st, int32_t max_calls) {
+  if (!st || !st->alive) return DGC_ESTATE;
+  if (max_calls < 0) return DGC_EINVAL;
+  DGC_CUDA(cudaSetDevice(st->device));
+  while ((int)st->prof_ev.size() < 2 * max_calls) {
+    cudaEvent_t e;
+    DGC_CUDA(cudaEventCreate(&e));
+    st->prof_ev.push_back(e);
+  }
+  st->prof_cap = max_calls;
+  st->prof_n = 0;
+  return DGC_OK;
+}
+
+int32_t dgc_profile_read(dgc_state* st, float* ms_out, int32_t capacity, int32_t* count_out) {
+  if (!st || !st->alive) return DGC_ESTATE;
+  if (!count_out || (capacity > 0 && !ms_out)) return DGC_EINVAL;
+  const int n = std::min<int>(st->prof_n, capacity);
+  for (int i = 0; i < n; ++i) {
+    DGC_CUDA(cudaEventSynchronize(st->prof_ev[2 * i + 1]));
+    DGC_CUDA(cudaEventElapsedTime(&ms_out[i], st->prof_ev[2 * i], st->prof_ev[2 * i + 1]));
+  }
+  *count_out = n;
   return DGC_OK;
 }
 
