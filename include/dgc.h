@@ -177,10 +177,13 @@ int32_t dgc_state_read(dgc_state* st, float* u_host, float* v_host, void* stream
 int32_t dgc_state_write(dgc_state* st, const float* u_host, const float* v_host, void* stream);
 
 /* Measurement aid (not part of the method): after dgc_profile_enable(st, n) the
- * next n dgc_compress calls record a CUDA event pair around their streaming
- * kernel (the fused Eq. 5 update + candidate emission pass) on the call's
- * stream.  dgc_profile_read waits for the recorded pairs and returns their
- * durations in milliseconds (ms_out[capacity], *count_out = pairs returned).
+ * next n dgc_compress calls record CUDA events on the call's stream at their
+ * stage boundaries.  dgc_profile_read waits for the recorded calls and returns,
+ * per call, five durations in milliseconds, ms_out[5 * call + stage]:
+ *   0 clipping norm   1 sampled threshold proposal   2 streaming pass (Eq. 5
+ *   update + candidate emission)   3 exact k-th key   4 ordered emission + masking
+ * (`capacity` = calls ms_out has room for; *count_out = calls returned).  A
+ * stage's duration includes the gap before its kernel starts.
  * dgc_profile_enable(st, 0) switches recording off. */
 int32_t dgc_profile_enable(dgc_state* st, int32_t max_calls);
 int32_t dgc_profile_read(dgc_state* st, float* ms_out, int32_t capacity, int32_t* count_out);

@@ -192,7 +192,8 @@ class State:
         _check(_lib.dgc_profile_enable(self._h, int(max_calls)), "dgc_profile_enable")
 
     def profile_read(self, capacity: int) -> np.ndarray:
-        ms = np.zeros(max(int(capacity), 1), np.float32)
+        """[calls, 5] stage durations in ms: norm, sample, streaming pass, select, emit."""
+        ms = np.zeros((max(int(capacity), 1), 5), np.float32)
         n = ctypes.c_int32()
         _check(_lib.dgc_profile_read(self._h, ms.ctypes.data, int(capacity), ctypes.byref(n)),
                "dgc_profile_read")

@@ -15,7 +15,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    deps = [SRC, os.path.join(INCLUDE, "dgc.h")]
+    deps = [SRC, os.path.join(_HERE, "csrc", "dgc_kernels.cuh"), os.path.join(INCLUDE, "dgc.h")]
     if (not force and os.path.exists(LIB)
             and all(os.path.getmtime(LIB) >= os.path.getmtime(d) for d in deps)):
         return LIB
@@ -27,4 +27,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    print(build(force=True, verbose="-v" in __import__("sys").argv))

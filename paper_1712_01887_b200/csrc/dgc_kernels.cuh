@@ -1,0 +1,1051 @@
+// sm_100a kernels of the Deep Gradient Compression hot path (device code only;
+// the host side and the C ABI are in dgc.cu).
+//
+// One dgc_compress call = one iteration of Algorithm 4 (Appendix D) on one
+// worker, as stream-ordered launches over a padded fp32 arena:
+//
+//   k_sumsq            (only when clipping)  Sec. 3.2 / App. C: ||g||_2 in fp64, coef
+//   k_sample_threshold Sec. 5: seeded sample of |v'| -> proposed threshold per tensor
+//   k_update_emit      Eq. 5: u' = m u + g coef, v' = v + u', stored once; entries whose
+//                      |v'| reaches the proposal are compacted, in index order per
+//                      512-element segment, into their part's candidate list
+//   k_select           exact k-th largest |v'| among a tensor's candidates (radix
+//                      select on the IEEE bit pattern), tie quota, per-part output bases
+//   k_emit_mask        Alg. 4 "G~ <- V (.) Mask", Sec. 3.3 masking: ordered (index, value)
+//                      pairs, then u = v = 0 at the sent entries
+//
+// The sample only proposes; if a proposal lets fewer than k_j entries or more
+// than the list capacity through, that tensor is selected from the whole of v'
+// instead (same result, slower).  All fp32 arithmetic uses explicit
+// round-to-nearest intrinsics so that no FMA contraction can change a bit.
+//
+// The tail kernels (sample, select, emit) touch little data; their cost is the
+// number of dependent global-memory round trips and block barriers on their
+// critical path, so tables are packed into 16/32-byte records fetched with one
+// load and the shared-memory phases are kept to two barriers per radix pass.
+//
+// Receive side: k_decode_bounds + k_decode_tiles (Alg. 4 aggregation line) and
+// k_sgd (Alg. 4 update line).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "dgc.h"
+
+namespace dgc {
+
+// ------------------------------------------------------------------ constants
+constexpr int kSeg = 512;              // elements per warp segment (4 x float4 per lane)
+constexpr int kPartSegs = 512;         // segments per part (256 Ki elements)
+constexpr int kSmallN = 8192;          // tensors up to this size are not sampled
+constexpr int kMaxSampleGroups = 8192; // float4 groups sampled per tensor at most
+constexpr int kSampleThreads = 512;    // one sampled float4 group per thread and block
+constexpr int kSampleSurvivors = 4096;
+constexpr int kSelectThreads = 1024;
+constexpr int kSelectMaxSmemKeys = 53248;
+constexpr int kSelectMaxParts = 1024;  // parts of one tensor whose tables fit in shared memory
+constexpr int kEmitThreads = kPartSegs;   // one thread per segment of the part
+constexpr int kEmitRegs = 8;              // candidates per thread kept in registers
+constexpr int kMaskStride = 17;           // words per segment in the winner bitmaps (16 + 1 pad)
+constexpr int kEmitSmemBytes = 2 * kPartSegs * kMaskStride * 4;
+constexpr int kMainThreads = 256;
+constexpr int kNormThreads = 256;
+constexpr int kMaxNormGrid = 2048;
+constexpr int kDecodeTile = 4096;
+constexpr int kDecodeThreads = 256;
+
+// ------------------------------------------------------------------ plan tables
+struct __align__(16) TensorMeta {   // one per tensor, read-only for the kernels
+  int32_t off, end;                 // arena range of the real elements
+  int32_t k, out_off;               // entries to send, first output slot
+  int32_t part_first, part_num;
+  int32_t rank, groups;             // sampling: rank of the proposal, float4 groups sampled
+  int32_t key_base, chunks;         // sampling: first key in the sample buffer, blocks that sample
+  int32_t pad0, pad1;
+};
+struct SampleBlock { int32_t tensor, chunk; };   // work item of one k_sample_threshold block
+struct __align__(16) PartMeta {     // one per part (up to kPartSegs segments of one tensor)
+  int32_t tensor, end;              // end: arena index one past the part's last real element
+  int32_t seg0, nseg;
+  int32_t cbase, cap;               // candidate list of the part
+  int32_t first, pad;               // first: this is the tensor's first part
+};
+struct __align__(16) PartSel {      // written by k_select, read by k_emit_mask
+  uint32_t kth;                     // bit pattern of the k-th largest |v'| of the tensor
+  int32_t quota;                    // entries tied with kth that this part sends
+  int32_t out_base;                 // first output slot of this part
+  int32_t dense;                    // 1: tensor takes the full-selection path
+};
+
+struct Plan {
+  const TensorMeta* tm;
+  const PartMeta* pm;
+  PartSel* psel;
+  int32_t* p_count;          // candidates appended per part (reset by k_emit_mask)
+  uint32_t* p_thr;           // proposed threshold per part (0 for tensors that are not sampled)
+  uint32_t* t_kth;           // per tensor: threshold of the last call (reporting)
+  int32_t* t_cand;           // per tensor: candidates of the last call, -1 = full selection
+  const int32_t* seg_part;   // part of every segment
+  const SampleBlock* sample_blocks;
+  uint32_t* sample_keys;     // |v'| keys of the current call's sample, all tensors
+  int32_t* sample_ticket;    // per tensor: sampling blocks that have finished
+  int32_t* cand_idx;
+  float* cand_val;
+  float* coef;
+  double* norm;
+  double* partials;
+  unsigned int* ticket;
+  long long* diag;           // [2][4]: flags, full_select, candidates, unused
+  float* u;
+  float* v;
+  int32_t num_tensors, num_parts, num_segs;
+};
+
+template <class T>
+__device__ __forceinline__ T load_record(const T* ptr) {
+  static_assert(sizeof(T) % 16 == 0, "records are whole int4s");
+  T out;
+  const int4* src = reinterpret_cast<const int4*>(ptr);
+  int4* dst = reinterpret_cast<int4*>(&out);
+#pragma unroll
+  for (int i = 0; i < (int)(sizeof(T) / 16); ++i) dst[i] = __ldcg(src + i);
+  return out;
+}
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+// Eq. 5, one element: gc = g*coef ; u <- m*u + gc ; v <- v + u (each rounded once).
+template <bool CLIP>
+__device__ __forceinline__ void mc_step(float g, float coef, float m, float& u, float& v) {
+  const float gc = CLIP ? __fmul_rn(g, coef) : g;
+  const float t = __fmul_rn(m, u);
+  u = __fadd_rn(t, gc);
+  v = __fadd_rn(v, u);
+}
+
+__device__ __forceinline__ uint64_t mix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+__device__ __forceinline__ int warp_incl_scan(int x) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xFFFFFFFFu, x, o);
+    if (lane >= o) x += t;
+  }
+  return x;
+}
+
+// Block-wide exclusive scan of two ints per thread (a, b); returns the
+// exclusive prefixes and the block totals.  `sh` needs 66 ints.  Two barriers;
+// a third is needed before `sh` is reused.
+__device__ __forceinline__ void block_excl_scan2(int a, int b, int* sh, int& ea, int& eb, int& ta,
+                                                 int& tb) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+  const int ia = warp_incl_scan(a), ib = warp_incl_scan(b);
+  if (lane == 31) { sh[warp] = ia; sh[33 + warp] = ib; }
+  __syncthreads();
+  if (warp == 0) {
+    const int wa = lane < nwarps ? sh[lane] : 0, wb = lane < nwarps ? sh[33 + lane] : 0;
+    const int sa = warp_incl_scan(wa), sb = warp_incl_scan(wb);
+    sh[lane] = sa - wa;
+    sh[33 + lane] = sb - wb;
+    if (lane == 31) { sh[32] = sa; sh[65] = sb; }
+  }
+  __syncthreads();
+  ea = sh[warp] + ia - a;
+  eb = sh[33 + warp] + ib - b;
+  ta = sh[32];
+  tb = sh[65];
+}
+
+// Radix select, descending: the `rank`-th largest key (rank >= 1) among the
+// keys the iterator visits.  `for_each(f)` must call f(valid, key) the same
+// number of times on every thread of the block (valid = false for padding
+// calls).  Every valid key lies in [base, maxkey]; only the bits in which
+// maxkey - base can differ are scanned, 8 per pass from the top.
+// hist: 512 words of shared memory (two 256-bin histograms, used alternately
+// so that one is cleared while the other is read), sh: 2 words.  The block
+// needs at least 288 threads.  Two barriers per pass plus one.
+// Returns the key; n_gt = number of keys strictly greater.
+constexpr int kHistWords = 512;
+
+template <class ForEach>
+__device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank, uint32_t base,
+                                                      uint32_t maxkey, uint32_t* hist, int* sh,
+                                                      int& n_gt) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  const uint32_t span = maxkey - base;
+  const int passes = span == 0 ? 0 : (32 - __clz(span) + 7) / 8;
+  uint32_t prefix = 0, mask = 0;
+  int remaining = rank;
+  if (tid < 256) hist[tid] = 0;
+  __syncthreads();
+  int cur = 0;
+  for (int shift = 8 * (passes - 1); shift >= 0; shift -= 8, cur ^= 1) {
+    uint32_t* h = hist + cur * 256;
+    for_each([&](bool valid, uint32_t key) {
+      key -= base;
+      uint32_t d = 0;
+      if (valid && (key & mask) == prefix) d = (key >> shift) & 255u; else valid = false;
+      // keys cluster on a few digits in the leading passes: lanes that share the digit of
+      // the first valid lane are added with one atomic, the others one by one
+      const unsigned vm = __ballot_sync(0xFFFFFFFFu, valid);
+      if (vm != 0) {
+        const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, d, __ffs(vm) - 1);
+        const unsigned m0 = __ballot_sync(0xFFFFFFFFu, valid && d == d0);
+        if (valid) {
+          if (d != d0) atomicAdd(&h[d], 1u);
+          else if (lane == __ffs(m0) - 1) atomicAdd(&h[d], (uint32_t)__popc(m0));
+        }
+      }
+    });
+    __syncthreads();
+    if (tid < 32) {
+      const int hi = 255 - 8 * lane;          // this lane covers bins hi, hi-1, .., hi-7
+      uint32_t loc[8];
+      uint32_t s = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { loc[q] = h[hi - q]; s += loc[q]; }
+      const uint32_t incl = (uint32_t)warp_incl_scan((int)s);
+      const uint32_t excl = incl - s;
+      if (excl < (uint32_t)remaining && (uint32_t)remaining <= incl) {
+        uint32_t c = excl;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (c + loc[q] >= (uint32_t)remaining) { sh[0] = hi - q; sh[1] = (int)c; break; }
+          c += loc[q];
+        }
+      }
+    } else if (tid < 288) {
+      hist[(cur ^ 1) * 256 + tid - 32] = 0;   // clear the other histogram for the next pass
+    }
+    __syncthreads();
+    prefix |= (uint32_t)sh[0] << shift;
+    mask |= 255u << shift;
+    remaining -= sh[1];
+  }
+  n_gt = rank - remaining;
+  return base + prefix;
+}
+
+// ------------------------------------------------------------------ K1: clipping norm
+// Sec. 3.2 / Appendix C.  Sum of squares of every real element of the gradient
+// set: fp32 loads, exact fp64 products, fp64 accumulation; fixed reduction
+// tree (grid size fixed per state), so the result does not depend on timing.
+// The last block to finish folds the partials and writes norm and coef.
+__global__ void __launch_bounds__(kNormThreads)
+k_sumsq(Plan p, const float* __restrict__ g, double thr_local, int clip_on) {
+  __shared__ double swarp[kNormThreads / 32];
+  __shared__ bool is_last;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int warps_total = gridDim.x * (kNormThreads / 32);
+  const float4* g4 = reinterpret_cast<const float4*>(g);
+  double acc = 0.0;
+  for (int seg = blockIdx.x * (kNormThreads / 32) + warp; seg < p.num_segs; seg += warps_total) {
+    const int base = seg * kSeg;
+    float4 x[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) x[i] = __ldg(g4 + (base >> 2) + i * 32 + lane);
+    const int part = __ldg(p.seg_part + seg);
+    const int end = __ldg(&p.pm[part].end);
+    if (base + kSeg <= end) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        acc += (double)x[i].x * (double)x[i].x;
+        acc += (double)x[i].y * (double)x[i].y;
+        acc += (double)x[i].z * (double)x[i].z;
+        acc += (double)x[i].w * (double)x[i].w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int e = base + (i * 32 + lane) * 4;
+        if (e + 0 < end) acc += (double)x[i].x * (double)x[i].x;
+        if (e + 1 < end) acc += (double)x[i].y * (double)x[i].y;
+        if (e + 2 < end) acc += (double)x[i].z * (double)x[i].z;
+        if (e + 3 < end) acc += (double)x[i].w * (double)x[i].w;
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+  if (lane == 0) swarp[warp] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w = 0; w < kNormThreads / 32; ++w) s += swarp[w];
+    p.partials[blockIdx.x] = s;
+    __threadfence();
+    const unsigned int t = atomicAdd(p.ticket, 1u);
+    is_last = (t == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // fold the per-block partials in a fixed order
+  double s = 0.0;
+  for (int i = threadIdx.x; i < (int)gridDim.x; i += kNormThreads) s += __ldcg(p.partials + i);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  if (lane == 0) swarp[warp] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double S = 0.0;
+    for (int w = 0; w < kNormThreads / 32; ++w) S += swarp[w];
+    const double norm = sqrt(S);
+    float coef = 1.0f;
+    if (clip_on && norm > thr_local) coef = (float)(thr_local / norm);
+    *p.norm = norm;
+    *p.coef = coef;
+    *p.ticket = 0u;
+  }
+}
+
+// ------------------------------------------------------------------ K2: sampled threshold proposal
+// Sec. 5: sample |v'| (v' computed on the fly from g, u, v exactly as the main
+// pass will), take the sample's rank-r key as the proposed threshold of the
+// tensor.  One float4 group per stratum at a hashed position.  The scattered
+// 16-byte loads are what costs, so a tensor's strata are spread over several
+// blocks (kSampleThreads groups each, one per thread); each block writes its
+// keys to a buffer and the last block of the tensor to finish (integer ticket)
+// selects.  r is small against the sample, so that block first bounds the
+// answer from below by the rank-r of the per-thread maxima (at least r keys
+// reach it), keeps the few keys that reach the bound and selects among them.
+template <bool CLIP>
+__global__ void __launch_bounds__(kSampleThreads)
+k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_seed) {
+  __shared__ uint32_t hist[kHistWords];
+  __shared__ uint32_t surv[kSampleSurvivors];
+  __shared__ int sh[2];
+  __shared__ int s_cnt;
+  __shared__ uint32_t s_max;
+  __shared__ int s_last;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const SampleBlock sb = p.sample_blocks[blockIdx.x];
+  const int j = sb.tensor;
+  const TensorMeta t = load_record(p.tm + j);
+  const int G = t.groups, rank = t.rank;
+  uint4* gkeys = reinterpret_cast<uint4*>(p.sample_keys + t.key_base);
+  {
+    const int s = sb.chunk * kSampleThreads + tid;
+    if (s < G) {
+      const uint32_t W = (uint32_t)((t.end - t.off) >> 2) / (uint32_t)G;   // groups per stratum
+      const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
+      // stratum s = groups [s*W, (s+1)*W); position inside it from a hash (multiply-high
+      // instead of a modulo); the < G groups after the last stratum are never sampled
+      const uint32_t h =
+          (uint32_t)mix64(call_seed ^ ((uint64_t)(uint32_t)j << 32) ^ (uint64_t)(uint32_t)s);
+      const uint32_t pos = (uint32_t)(t.off >> 2) + (uint32_t)s * W + __umulhi(h, W);
+      const float4 gg = __ldg(reinterpret_cast<const float4*>(g) + pos);
+      float4 u = __ldcg(reinterpret_cast<const float4*>(p.u) + pos);
+      float4 v = __ldcg(reinterpret_cast<const float4*>(p.v) + pos);
+      mc_step<CLIP>(gg.x, coef, m, u.x, v.x);
+      mc_step<CLIP>(gg.y, coef, m, u.y, v.y);
+      mc_step<CLIP>(gg.z, coef, m, u.z, v.z);
+      mc_step<CLIP>(gg.w, coef, m, u.w, v.w);
+      gkeys[s] = make_uint4(mag_key(v.x), mag_key(v.y), mag_key(v.z), mag_key(v.w));
+    }
+  }
+  if (t.chunks > 1) {
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+      const int done = atomicAdd(p.sample_ticket + j, 1);
+      s_last = done == t.chunks - 1;
+      if (s_last) p.sample_ticket[j] = 0;       // ready for the next call
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+  }
+  if (tid == 0) { s_cnt = 0; s_max = 0u; }
+  __syncthreads();                                    // also orders this block's own key writes
+  // this block now holds the whole sample of the tensor in gkeys[0 .. G)
+  const int iters = (G + kSampleThreads - 1) / kSampleThreads;
+  uint32_t tmax = 0;
+#pragma unroll 4
+  for (int it = 0; it < iters; ++it) {
+    const int i = it * kSampleThreads + tid;
+    if (i < G) {
+      const uint4 kk = __ldcg(gkeys + i);
+      tmax = max(max(tmax, kk.x), max(kk.y, max(kk.z, kk.w)));
+    }
+  }
+  {
+    const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
+    if (lane == 0) atomicMax(&s_max, wmax);
+  }
+  __syncthreads();
+  const uint32_t kmax = s_max;
+  const int owners = min(G, kSampleThreads);          // threads that hold at least one group
+  int n_gt;
+  uint32_t kth = 0;
+  bool done = false;
+  if (rank <= owners) {
+    // lower bound: rank-th largest of the thread maxima
+    const uint32_t low = block_select_desc([&](auto f) { f(tid < owners, tmax); }, rank, 0u, kmax,
+                                           hist, sh, n_gt);
+    // keep the keys that reach it
+#pragma unroll 4
+    for (int it = 0; it < iters; ++it) {
+      const int i = it * kSampleThreads + tid;
+      uint4 kk = make_uint4(0u, 0u, 0u, 0u);
+      if (i < G) kk = __ldcg(gkeys + i);
+      const uint32_t karr[4] = {kk.x, kk.y, kk.z, kk.w};
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const bool keep = i < G && karr[c] >= low;
+        const unsigned mk = __ballot_sync(0xFFFFFFFFu, keep);
+        if (mk) {
+          int basepos = 0;
+          if (lane == __ffs(mk) - 1) basepos = atomicAdd(&s_cnt, __popc(mk));
+          basepos = __shfl_sync(0xFFFFFFFFu, basepos, __ffs(mk) - 1);
+          const int pos = basepos + __popc(mk & ((1u << lane) - 1u));
+          if (keep && pos < kSampleSurvivors) surv[pos] = karr[c];
+        }
+      }
+    }
+    __syncthreads();
+    const int ns = s_cnt;
+    if (ns <= kSampleSurvivors) {
+      const int it2 = (ns + kSampleThreads - 1) / kSampleThreads;
+      kth = block_select_desc(
+          [&](auto f) {
+            for (int it = 0; it < it2; ++it) {
+              const int i = it * kSampleThreads + tid;
+              f(i < ns, i < ns ? surv[i] : low);
+            }
+          },
+          rank, low, kmax, hist, sh, n_gt);
+      done = true;
+    }
+  }
+  if (!done) {
+    kth = block_select_desc(
+        [&](auto f) {
+          for (int it = 0; it < iters; ++it) {
+            const int i = it * kSampleThreads + tid;
+            uint4 kk = make_uint4(0u, 0u, 0u, 0u);
+            if (i < G) kk = __ldcg(gkeys + i);
+            f(i < G, kk.x);
+            f(i < G, kk.y);
+            f(i < G, kk.z);
+            f(i < G, kk.w);
+          }
+        },
+        rank, 0u, kmax, hist, sh, n_gt);
+  }
+  // a proposal of 0 would let every entry through: insist on non-zero magnitude
+  const uint32_t thr = kth > 1u ? kth : 1u;
+  for (int q = tid; q < t.part_num; q += kSampleThreads) p.p_thr[t.part_first + q] = thr;
+}
+
+// ------------------------------------------------------------------ K3: fused momentum correction + candidate emission
+// The streaming pass: 12 B read + 8 B written per element.  Each warp owns one
+// 512-element segment at a time (4 float4 per lane per array, 512 contiguous
+// bytes per warp load), keeps everything in registers, and appends the
+// segment's candidates -- in ascending index order -- to its part's list with
+// one integer atomicAdd per segment that has any.
+template <bool CLIP>
+__global__ void __launch_bounds__(kMainThreads)
+k_update_emit(Plan p, const float* __restrict__ g, float m) {
+  const int lane = threadIdx.x & 31;
+  const float4* g4 = reinterpret_cast<const float4*>(g);
+  float4* u4 = reinterpret_cast<float4*>(p.u);
+  float4* v4 = reinterpret_cast<float4*>(p.v);
+  // one segment per warp, one launch-time block per 8 segments: short blocks let the
+  // hardware interleave this kernel with the small kernels of other streams
+  const int seg = blockIdx.x * (kMainThreads / 32) + (threadIdx.x >> 5);
+  if (seg < p.num_segs) {
+    const int base = seg * kSeg;
+    const int q0 = (base >> 2) + lane;
+    float4 gg[4], uu[4], vv[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) gg[i] = __ldcs(g4 + q0 + i * 32);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) uu[i] = __ldcs(u4 + q0 + i * 32);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) vv[i] = __ldcs(v4 + q0 + i * 32);
+    const int part = __ldg(p.seg_part + seg);
+    const PartMeta pm = load_record(p.pm + part);
+    const uint32_t thr = __ldcg(p.p_thr + part);
+    const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
+    const int end = pm.end;
+    const bool full = base + kSeg <= end;
+    uint32_t flags = 0;   // bit (4*i + c): element c of float4 i is a candidate
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      mc_step<CLIP>(gg[i].x, coef, m, uu[i].x, vv[i].x);
+      mc_step<CLIP>(gg[i].y, coef, m, uu[i].y, vv[i].y);
+      mc_step<CLIP>(gg[i].z, coef, m, uu[i].z, vv[i].z);
+      mc_step<CLIP>(gg[i].w, coef, m, uu[i].w, vv[i].w);
+      flags |= (uint32_t)(mag_key(vv[i].x) >= thr) << (4 * i + 0);
+      flags |= (uint32_t)(mag_key(vv[i].y) >= thr) << (4 * i + 1);
+      flags |= (uint32_t)(mag_key(vv[i].z) >= thr) << (4 * i + 2);
+      flags |= (uint32_t)(mag_key(vv[i].w) >= thr) << (4 * i + 3);
+    }
+    if (full) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) __stcs(u4 + q0 + i * 32, uu[i]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) __stcs(v4 + q0 + i * 32, vv[i]);
+    } else {
+      // ragged end of a tensor: only real elements are stored or can be candidates
+      uint32_t valid = 0;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int e = base + (i * 32 + lane) * 4;
+        const float uarr[4] = {uu[i].x, uu[i].y, uu[i].z, uu[i].w};
+        const float varr[4] = {vv[i].x, vv[i].y, vv[i].z, vv[i].w};
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          if (e + c < end) {
+            valid |= 1u << (4 * i + c);
+            p.u[e + c] = uarr[c];
+            p.v[e + c] = varr[c];
+          }
+        }
+      }
+      flags &= valid;
+    }
+    if (__any_sync(0xFFFFFFFFu, flags != 0)) {
+      // per-lane counts of the four float4 rows packed one per byte (row totals <= 128)
+      const uint32_t cnt = __popc(flags & 0xFu) | (__popc(flags & 0xF0u) << 8) |
+                           (__popc(flags & 0xF00u) << 16) | (__popc(flags & 0xF000u) << 24);
+      const uint32_t incl = (uint32_t)warp_incl_scan((int)cnt);
+      const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+      const uint32_t excl = incl - cnt;
+      const int t0 = tot & 255, t1 = (tot >> 8) & 255, t2 = (tot >> 16) & 255, t3 = tot >> 24;
+      const int seg_total = t0 + t1 + t2 + t3;
+      int start = 0;
+      if (lane == 0) start = atomicAdd(p.p_count + part, seg_total);
+      start = __shfl_sync(0xFFFFFFFFu, start, 0);
+      const int row_base[4] = {0, t0, t0 + t1, t0 + t1 + t2};
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t nib = (flags >> (4 * i)) & 0xFu;
+        if (nib) {
+          int pos = start + row_base[i] + (int)((excl >> (8 * i)) & 255u);
+          const int e = base + (i * 32 + lane) * 4;
+          const float varr[4] = {vv[i].x, vv[i].y, vv[i].z, vv[i].w};
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            if (nib & (1u << c)) {
+              if (pos < pm.cap) {
+                p.cand_idx[pm.cbase + pos] = e + c;
+                p.cand_val[pm.cbase + pos] = varr[c];
+              }
+              ++pos;
+            }
+          }
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------ K4: exact k-th key per tensor
+// Algorithm 4 "thr <- s% of |V[j]|" made exact: the k_j-th largest |v'| among
+// the tensor's candidates, the number of strictly larger ones and the tie
+// quota; then each part's first output slot and its share of the ties (ties go
+// to the lower index, so to the earlier part).  One block per tensor.
+__global__ void __launch_bounds__(kSelectThreads)
+k_select(Plan p, int smem_keys, int parity) {
+  extern __shared__ uint32_t skeys[];
+  __shared__ uint32_t hist[kHistWords];
+  __shared__ int sh[66];
+  __shared__ int s_flag;
+  __shared__ uint32_t s_max;
+  __shared__ int s_pbase[kSelectMaxParts + 1];   // first key of each part in the compact order
+  __shared__ int s_pcb[kSelectMaxParts];         // start of each part's candidate list
+  __shared__ int s_gt[kSelectMaxParts];
+  __shared__ int s_eq[kSelectMaxParts];
+  const int j = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const TensorMeta t = load_record(p.tm + j);
+  const int p0 = t.part_first, pn = t.part_num, k = t.k;
+  const bool tables = pn <= kSelectMaxParts;
+  if (j == 0 && tid < 4) p.diag[(parity ^ 1) * 4 + tid] = 0;   // next call's counters
+  if (tid == 0) { s_flag = 0; s_max = 0u; }
+  __syncthreads();
+  // candidates per part (one load round for all parts), overflow check, compact bases
+  int total = 0;
+  if (pn <= 32) {
+    if (warp == 0) {
+      int c = 0;
+      if (lane < pn) {
+        const PartMeta pm = load_record(p.pm + p0 + lane);
+        c = __ldcg(p.p_count + p0 + lane);
+        if (c > pm.cap) s_flag = 1;
+        s_pcb[lane] = pm.cbase;
+      }
+      const int incl = warp_incl_scan(c);
+      if (lane < pn) s_pbase[lane] = incl - c;
+      if (lane == 31) s_pbase[pn] = incl;
+    }
+    __syncthreads();
+    total = s_pbase[pn];
+  } else {
+    for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+      const int q = q0 + tid;
+      int c = 0;
+      if (q < pn) {
+        const PartMeta pm = load_record(p.pm + p0 + q);
+        c = __ldcg(p.p_count + p0 + q);
+        if (c > pm.cap) s_flag = 1;
+        if (tables) s_pcb[q] = pm.cbase;
+      }
+      int ex, dummy_e, tot, dummy_t;
+      block_excl_scan2(c, 0, sh, ex, dummy_e, tot, dummy_t);
+      if (tables && q < pn) s_pbase[q] = total + ex;
+      total += tot;
+      __syncthreads();
+    }
+    if (tables && tid == 0) s_pbase[pn] = total;
+    __syncthreads();
+  }
+  const bool overflow = s_flag != 0;
+  if (overflow || total < k) {
+    // full-selection path: k_emit_mask's block of the tensor's first part does it
+    for (int q = tid; q < pn; q += kSelectThreads) {
+      PartSel ps;
+      ps.kth = 0u; ps.quota = 0; ps.out_base = 0; ps.dense = 1;
+      p.psel[p0 + q] = ps;
+    }
+    if (tid == 0) {
+      p.t_cand[j] = -1;
+      atomicOr((unsigned long long*)&p.diag[parity * 4 + 0],
+               (unsigned long long)(DGC_FLAG_FULL_SELECT |
+                                    (overflow ? DGC_FLAG_CAND_OVERFLOW : DGC_FLAG_CAND_SHORT)));
+      atomicAdd((unsigned long long*)&p.diag[parity * 4 + 1], 1ull);
+    }
+    return;
+  }
+  const bool in_smem = tables && total <= smem_keys;
+  uint32_t kmax = 0x7FFFFFFFu;
+  uint32_t kbase = 0u;
+  if (in_smem) {
+    // gather the keys of all parts, compact, into shared memory: every load independent
+    uint32_t tmax = 0;
+#pragma unroll 4
+    for (int i = tid; i < total; i += kSelectThreads) {
+      int lo = 0, hi = pn;                       // largest q with s_pbase[q] <= i
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (s_pbase[mid] <= i) lo = mid; else hi = mid;
+      }
+      const uint32_t key = mag_key(__ldcg(p.cand_val + s_pcb[lo] + (i - s_pbase[lo])));
+      skeys[i] = key;
+      tmax = max(tmax, key);
+    }
+    const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
+    if (lane == 0) atomicMax(&s_max, wmax);
+    kbase = __ldcg(p.p_thr + p0);                // every candidate reached the proposal
+    __syncthreads();
+    kmax = s_max;
+  }
+  int n_gt;
+  uint32_t kth;
+  if (in_smem) {
+    const int iters = (total + kSelectThreads - 1) / kSelectThreads;
+    kth = block_select_desc(
+        [&](auto f) {
+          for (int it = 0; it < iters; ++it) {
+            const int i = it * kSelectThreads + tid;
+            const bool valid = i < total;
+            f(valid, valid ? skeys[i] : kbase);
+          }
+        },
+        k, kbase, kmax, hist, sh, n_gt);
+  } else {
+    kth = block_select_desc(
+        [&](auto f) {
+          for (int q = 0; q < pn; ++q) {
+            const int c = __ldcg(p.p_count + p0 + q);
+            const float* src = p.cand_val + __ldg(&p.pm[p0 + q].cbase);
+            const int iters = (c + kSelectThreads - 1) / kSelectThreads;
+            for (int it = 0; it < iters; ++it) {
+              const int i = it * kSelectThreads + tid;
+              const bool valid = i < c;
+              f(valid, valid ? mag_key(__ldcg(src + i)) : 0u);
+            }
+          }
+        },
+        k, kbase, kmax, hist, sh, n_gt);
+  }
+  const int quota = k - n_gt;   // ties (|v'| == kth) to take, lowest indices first
+  const int out_off = t.out_off;
+  if (tables) {
+    // per part: strictly-greater and tied candidates; one warp per part
+    for (int q = warp; q < pn; q += kSelectThreads / 32) {
+      int gt = 0, eq = 0;
+      if (in_smem) {
+        const int b0 = s_pbase[q], b1 = s_pbase[q + 1];
+        for (int i = b0 + lane; i < b1; i += 32) {
+          const uint32_t key = skeys[i];
+          gt += key > kth;
+          eq += key == kth;
+        }
+      } else {
+        const int c = s_pbase[q + 1] - s_pbase[q];
+        const float* src = p.cand_val + s_pcb[q];
+        for (int i = lane; i < c; i += 32) {
+          const uint32_t key = mag_key(__ldcg(src + i));
+          gt += key > kth;
+          eq += key == kth;
+        }
+      }
+      gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+      eq = __reduce_add_sync(0xFFFFFFFFu, eq);
+      if (lane == 0) { s_gt[q] = gt; s_eq[q] = eq; }
+    }
+    __syncthreads();
+    if (pn <= 32) {
+      if (warp == 0) {
+        const int gt = lane < pn ? s_gt[lane] : 0, eq = lane < pn ? s_eq[lane] : 0;
+        const int bg = warp_incl_scan(gt) - gt, be = warp_incl_scan(eq) - eq;
+        if (lane < pn) {
+          PartSel ps;
+          ps.kth = kth;
+          ps.quota = max(0, min(quota - be, eq));
+          ps.out_base = out_off + bg + min(be, quota);
+          ps.dense = 0;
+          p.psel[p0 + lane] = ps;
+        }
+      }
+    } else {
+      int run_gt = 0, run_eq = 0;
+      for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+        const int q = q0 + tid;
+        const int gt = q < pn ? s_gt[q] : 0, eq = q < pn ? s_eq[q] : 0;
+        int bg, be, tg, te;
+        block_excl_scan2(gt, eq, sh, bg, be, tg, te);
+        bg += run_gt;
+        be += run_eq;
+        if (q < pn) {
+          PartSel ps;
+          ps.kth = kth;
+          ps.quota = max(0, min(quota - be, eq));
+          ps.out_base = out_off + bg + min(be, quota);
+          ps.dense = 0;
+          p.psel[p0 + q] = ps;
+        }
+        run_gt += tg;
+        run_eq += te;
+        __syncthreads();
+      }
+    }
+  } else {
+    // more parts than the tables hold: walk them in chunks, counting from global memory
+    int run_gt = 0, run_eq = 0;
+    for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+      const int q = q0 + tid;
+      int gt = 0, eq = 0;
+      if (q < pn) {
+        const int c = __ldcg(p.p_count + p0 + q);
+        const float* src = p.cand_val + __ldg(&p.pm[p0 + q].cbase);
+        for (int i = 0; i < c; ++i) {
+          const uint32_t key = mag_key(__ldcg(src + i));
+          gt += key > kth;
+          eq += key == kth;
+        }
+      }
+      int bg, be, tg, te;
+      block_excl_scan2(gt, eq, sh, bg, be, tg, te);
+      bg += run_gt;
+      be += run_eq;
+      if (q < pn) {
+        PartSel ps;
+        ps.kth = kth;
+        ps.quota = max(0, min(quota - be, eq));
+        ps.out_base = out_off + bg + min(be, quota);
+        ps.dense = 0;
+        p.psel[p0 + q] = ps;
+      }
+      run_gt += tg;
+      run_eq += te;
+      __syncthreads();
+    }
+  }
+  if (tid == 0) {
+    p.t_kth[j] = kth;
+    p.t_cand[j] = total;
+    atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
+  }
+}
+
+// ------------------------------------------------------------------ K5: ordered emission + masking
+// Algorithm 4: G~[j] <- V[j] (.) Mask ; V[j] <- V[j] (.) !Mask ; U[j] <- U[j] (.) !Mask.
+// One block per part.  The candidates that reach the threshold set one bit
+// each in a shared-memory bitmap of the part (integer atomicOr; "greater" and
+// "tied" bitmaps); per-segment popcounts and an exclusive scan give every
+// segment its first output slot; every winner then finds its slot from the
+// bits below its own, writes its (index, value) pair and zeroes u and v there.
+//
+// Full-selection path (dense flag set by k_select): the block of the tensor's
+// first part selects from the whole of v' (radix select over global memory) and
+// emits by walking the tensor in order.  Same result; slow; rare.
+__device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int32_t* out_idx,
+                                  float* out_val, uint32_t* hist, int* sh) {
+  const int tid = threadIdx.x, nt = blockDim.x;
+  const int off = t.off;
+  const int n = t.end - off;
+  const int k = t.k;
+  const float* v = p.v + off;
+  const int iters = (n + nt - 1) / nt;
+  int n_gt;
+  const uint32_t kth = block_select_desc(
+      [&](auto f) {
+        for (int it = 0; it < iters; ++it) {
+          const int i = it * nt + tid;
+          const bool valid = i < n;
+          f(valid, valid ? mag_key(__ldcg(v + i)) : 0u);
+        }
+      },
+      k, 0u, 0x7FFFFFFFu, hist, sh, n_gt);
+  const int quota = k - n_gt;
+  int run_w = 0, run_eq = 0;     // winners / ties seen so far
+  for (int c0 = 0; c0 < n; c0 += nt * 4) {
+    const int e0 = c0 + tid * 4;
+    float x[4];
+    int gt = 0, eq = 0;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      x[c] = (e0 + c < n) ? __ldcg(v + e0 + c) : 0.0f;
+      const uint32_t key = mag_key(x[c]);
+      if (e0 + c < n) { gt += key > kth; eq += key == kth; }
+    }
+    int bg, be, tg, te;
+    block_excl_scan2(gt, eq, sh, bg, be, tg, te);
+    be += run_eq;
+    int pos = t.out_off + run_w + bg + (min(be, quota) - min(run_eq, quota));
+    int eqr = be;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      if (e0 + c < n) {
+        const uint32_t key = mag_key(x[c]);
+        bool take = key > kth;
+        if (key == kth) { take = eqr < quota; ++eqr; }
+        if (take) {
+          out_idx[pos] = off + e0 + c;
+          out_val[pos] = x[c];
+          p.u[off + e0 + c] = 0.0f;
+          p.v[off + e0 + c] = 0.0f;
+          ++pos;
+        }
+      }
+    }
+    run_w += tg + (min(run_eq + te, quota) - min(run_eq, quota));
+    run_eq += te;
+    __syncthreads();
+  }
+  if (tid == 0) p.t_kth[j] = kth;
+}
+
+__global__ void __launch_bounds__(kEmitThreads)
+k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
+  extern __shared__ uint32_t smask[];          // winner bitmaps of the part: [gt | eq]
+  __shared__ int sh[66];
+  __shared__ int s_gtb[kPartSegs];             // winners before each segment
+  __shared__ int s_eqb[kPartSegs];
+  static_assert(kEmitSmemBytes >= kHistWords * 4, "bitmaps double as histograms");
+  uint32_t* mgt = smask;
+  uint32_t* meq = smask + kPartSegs * kMaskStride;
+  const int part = blockIdx.x;
+  const int tid = threadIdx.x;
+  // one round of independent loads: part record, selection result, candidate count
+  const PartMeta pm = load_record(p.pm + part);
+  const PartSel ps = load_record(p.psel + part);
+  const int count = __ldcg(p.p_count + part);
+  if (ps.dense) {
+    __syncthreads();
+    if (tid == 0) p.p_count[part] = 0;
+    if (pm.first) {
+      const TensorMeta t = load_record(p.tm + pm.tensor);
+      dense_select_emit(p, t, pm.tensor, out_idx, out_val, smask, sh);
+    }
+    return;
+  }
+  const uint32_t kth = ps.kth;
+  const int quota = ps.quota;
+  const int32_t* cidx = p.cand_idx + pm.cbase;
+  const float* cval = p.cand_val + pm.cbase;
+  // first kEmitRegs candidates of every thread stay in registers
+  float vals[kEmitRegs];
+#pragma unroll
+  for (int b = 0; b < kEmitRegs; ++b) {
+    const int i = b * kEmitThreads + tid;
+    vals[b] = i < count ? __ldcg(cval + i) : 0.0f;
+  }
+  for (int i = tid; i < 2 * kPartSegs * kMaskStride; i += kEmitThreads) smask[i] = 0u;
+  __syncthreads();
+  if (tid == 0) p.p_count[part] = 0;          // ready for the next call
+  // mark the candidates that reach the threshold: one bit per element of the part
+  int locs[kEmitRegs];
+#pragma unroll
+  for (int b = 0; b < kEmitRegs; ++b) {
+    const int i = b * kEmitThreads + tid;
+    const uint32_t key = mag_key(vals[b]);
+    locs[b] = -1;
+    if (i < count && key >= kth) {
+      const int local = __ldcg(cidx + i) - pm.seg0 * kSeg;
+      locs[b] = local;
+      const int word = (local >> 9) * kMaskStride + ((local >> 5) & 15);
+      atomicOr((key > kth ? mgt : meq) + word, 1u << (local & 31));
+    }
+  }
+  for (int i = kEmitRegs * kEmitThreads + tid; i < count; i += kEmitThreads) {
+    const uint32_t key = mag_key(__ldcg(cval + i));
+    if (key >= kth) {
+      const int local = __ldcg(cidx + i) - pm.seg0 * kSeg;
+      const int word = (local >> 9) * kMaskStride + ((local >> 5) & 15);
+      atomicOr((key > kth ? mgt : meq) + word, 1u << (local & 31));
+    }
+  }
+  __syncthreads();
+  // thread s owns segment s: popcounts, then winners before each segment
+  {
+    int gt = 0, eq = 0;
+    if (tid < pm.nseg) {
+#pragma unroll
+      for (int w = 0; w < 16; ++w) {
+        gt += __popc(mgt[tid * kMaskStride + w]);
+        eq += __popc(meq[tid * kMaskStride + w]);
+      }
+    }
+    int bg, be, tg, te;
+    block_excl_scan2(gt, eq, sh, bg, be, tg, te);
+    s_gtb[tid] = bg;
+    s_eqb[tid] = be;
+  }
+  __syncthreads();
+  auto emit = [&](int local, float val, uint32_t key) {
+    const int s = local >> 9, w = (local >> 5) & 15;
+    const uint32_t below = (1u << (local & 31)) - 1u;
+    int lg = __popc(mgt[s * kMaskStride + w] & below);
+    int le = __popc(meq[s * kMaskStride + w] & below);
+    for (int x = 0; x < w; ++x) {
+      lg += __popc(mgt[s * kMaskStride + x]);
+      le += __popc(meq[s * kMaskStride + x]);
+    }
+    const int eq_before = s_eqb[s] + le;         // ties with a lower index, whole part
+    int pos;
+    if (key > kth) {
+      pos = ps.out_base + s_gtb[s] + lg + min(eq_before, quota);
+    } else {
+      if (eq_before >= quota) return;            // ties: lowest indices first
+      pos = ps.out_base + s_gtb[s] + lg + eq_before;
+    }
+    const int idx = pm.seg0 * kSeg + local;
+    out_idx[pos] = idx;
+    out_val[pos] = val;
+    p.u[idx] = 0.0f;
+    p.v[idx] = 0.0f;
+  };
+#pragma unroll
+  for (int b = 0; b < kEmitRegs; ++b)
+    if (locs[b] >= 0) emit(locs[b], vals[b], mag_key(vals[b]));
+  for (int i = kEmitRegs * kEmitThreads + tid; i < count; i += kEmitThreads) {
+    const float val = __ldcg(cval + i);
+    const uint32_t key = mag_key(val);
+    if (key >= kth) emit(__ldcg(cidx + i) - pm.seg0 * kSeg, val, key);
+  }
+}
+
+// ------------------------------------------------------------------ receive side
+// Alg. 4 "G_t <- sum_k encode(G~_k)".  k_decode_bounds finds, for every worker
+// list (ascending indices), where each tile of the dense output starts;
+// k_decode_tiles accumulates a tile in shared memory one worker after the other
+// (indices within one worker are unique, so no two threads touch one slot
+// between barriers) and writes it once.
+struct DecodeArgs {
+  const int32_t* idx[DGC_MAX_DECODE_WORKERS];
+  const float* val[DGC_MAX_DECODE_WORKERS];
+  int32_t nnz[DGC_MAX_DECODE_WORKERS];
+  int32_t num_workers;
+  int32_t num_tiles;
+};
+
+__global__ void __launch_bounds__(256)
+k_decode_bounds(const __grid_constant__ DecodeArgs a, int32_t* __restrict__ bounds) {
+  // bounds[w * (num_tiles + 1) + t] = first position in list w whose index >= t * tile
+  const int w = blockIdx.y;
+  const int n = a.nnz[w];
+  const int32_t* idx = a.idx[w];
+  int32_t* b = bounds + (size_t)w * (a.num_tiles + 1);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i <= n; i += gridDim.x * blockDim.x) {
+    const int t_prev = (i == 0) ? -1 : (__ldg(idx + i - 1) / kDecodeTile);
+    const int t_cur = (i == n) ? a.num_tiles : (__ldg(idx + i) / kDecodeTile);
+    for (int t = t_prev + 1; t <= t_cur; ++t) b[t] = i;
+  }
+}
+
+__global__ void __launch_bounds__(kDecodeThreads)
+k_decode_tiles(const __grid_constant__ DecodeArgs a, const int32_t* __restrict__ bounds,
+               float* __restrict__ dense, long long dense_len) {
+  __shared__ float tile[kDecodeTile];
+  __shared__ int s_lo[DGC_MAX_DECODE_WORKERS], s_hi[DGC_MAX_DECODE_WORKERS];
+  const int t = blockIdx.x;
+  const long long base = (long long)t * kDecodeTile;
+  if (threadIdx.x < a.num_workers) {
+    const int32_t* b = bounds + (size_t)threadIdx.x * (a.num_tiles + 1);
+    s_lo[threadIdx.x] = __ldg(b + t);
+    s_hi[threadIdx.x] = __ldg(b + t + 1);
+  }
+#pragma unroll
+  for (int i = threadIdx.x; i < kDecodeTile; i += kDecodeThreads) tile[i] = 0.0f;
+  __syncthreads();
+  for (int w = 0; w < a.num_workers; ++w) {
+    const int lo = s_lo[w], hi = s_hi[w];
+    if (hi > lo) {      // block-uniform
+      const int32_t* idx = a.idx[w];
+      const float* val = a.val[w];
+      for (int i = lo + threadIdx.x; i < hi; i += kDecodeThreads) {
+        const int l = __ldg(idx + i) - (int)base;
+        tile[l] = __fadd_rn(tile[l], __ldg(val + i));
+      }
+      __syncthreads();
+    }
+  }
+  const long long rem = dense_len - base;
+  if (rem >= kDecodeTile) {
+    float4* d4 = reinterpret_cast<float4*>(dense + base);
+    const float4* t4 = reinterpret_cast<const float4*>(tile);
+#pragma unroll
+    for (int i = threadIdx.x; i < kDecodeTile / 4; i += kDecodeThreads) __stcs(d4 + i, t4[i]);
+  } else {
+    for (int i = threadIdx.x; i < (int)rem; i += kDecodeThreads) dense[base + i] = tile[i];
+  }
+}
+
+// Alg. 4 "theta <- SGD(theta, G_t)": w <- w - lr*G, two roundings.
+__global__ void __launch_bounds__(256)
+k_sgd(float* __restrict__ w, const float* __restrict__ G, long long len, float lr) {
+  const long long n4 = len >> 2;
+  float4* w4 = reinterpret_cast<float4*>(w);
+  const float4* g4 = reinterpret_cast<const float4*>(G);
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+    float4 a = __ldcs(w4 + i);
+    const float4 b = __ldcs(g4 + i);
+    a.x = __fsub_rn(a.x, __fmul_rn(lr, b.x));
+    a.y = __fsub_rn(a.y, __fmul_rn(lr, b.y));
+    a.z = __fsub_rn(a.z, __fmul_rn(lr, b.z));
+    a.w = __fsub_rn(a.w, __fmul_rn(lr, b.w));
+    __stcs(w4 + i, a);
+  }
+  if (blockIdx.x == 0 && threadIdx.x < (int)(len & 3)) {
+    const long long i = (n4 << 2) + threadIdx.x;
+    w[i] = __fsub_rn(w[i], __fmul_rn(lr, G[i]));
+  }
+}
+
+}  // namespace dgc
