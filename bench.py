@@ -41,6 +41,9 @@ METRIC = "compressed gradient elements/s"
 UNIT = "elements/s"
 POOL = 2            # distinct pre-generated gradients per worker
 LR = 0.01
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_update_emit launch, from the ncu capture
+# summarised in profiles/k_update_emit_resnet50_ncu_full.md (same per-launch size as the bench)
+NCU_TRAFFIC_BYTES = {"resnet50": 307.19e6 + 151.20e6}
 
 
 def _peaks():
@@ -300,7 +303,9 @@ def run_ours(args):
                      "kernel_timing": "CUDA events around the kernel inside dgc_compress, on its "
                                       "stream, in an instrumented single-stream repeat of the "
                                       "same K steps",
-                     "algorithmic_bytes_per_launch": alg_bytes, "traffic": args.traffic},
+                     "algorithmic_bytes_per_launch": alg_bytes,
+                     "traffic": args.traffic if args.traffic is not None
+                     else NCU_TRAFFIC_BYTES.get(wl.name)},
         "stages_ms": dict(zip(["norm", "sample", "stream", "select", "emit"],
                               [float(x) for x in stage_ms.mean(axis=0)])),
         "compress": {"ms_per_worker": compress_ms, "elements_per_s": total / (compress_ms * 1e-3),
