@@ -42,6 +42,7 @@ extern "C" {
 
 #define DGC_ARENA_ALIGN        512   /* elements; tensor starts and arena length */
 #define DGC_MAX_DECODE_WORKERS 64
+#define DGC_STATIC_DECODE_WORDS (1 << 18)   /* int32 words of built-in decode scratch (1 MiB) */
 
 /* dgc_status.flags */
 #define DGC_FLAG_NONFINITE_NORM   1  /* the clipping norm was Inf or NaN            */
@@ -156,6 +157,30 @@ int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lis
                               int64_t dense_len, void* workspace, int64_t workspace_bytes,
                               void* stream);
 int64_t dgc_decode_workspace_bytes(int32_t num_workers, int64_t dense_len);
+
+/* The paper has no counterpart to this call: it is dgc_decode_accumulate for callers that
+ * must not allocate device memory.  Two kinds of caller are meant.  One runs inside a
+ * framework whose caching allocator has already claimed the whole GPU, so a raw cudaMalloc
+ * for a workspace would fail or force the cache to be flushed.  The other sits in a
+ * latency-critical loop (a serving step, a training inner loop), where cudaMalloc and cudaFree
+ * are off limits because they synchronise the whole device.  Such callers still pass their
+ * inputs and the output buffer, but no workspace: the tile-boundary scratch is a fixed
+ * DGC_STATIC_DECODE_WORDS * 4 byte (1 MiB) array built into the library, which every GPU that
+ * loads the library carries until the process exits.  The call itself performs no cudaMalloc,
+ * cudaFree or other allocating call.
+ *   Same arguments, result and preconditions as dgc_decode_accumulate (dense_out is bit for
+ * bit the same), minus `workspace`.  Limit: num_workers * (ceil(dense_len / 4096) + 1) must
+ * not exceed DGC_STATIC_DECODE_WORDS (e.g. 8 workers up to 134 M dense elements); a larger
+ * problem returns DGC_ECAPACITY and enqueues nothing.
+ *   The first call on each device looks up the array's device address (the device that is
+ * current at that call must be the one that owns the buffers); make that first call before
+ * starting any stream capture.  All calls on a device share the one array: it still holds the
+ * previous call's boundaries, which is harmless because every word a call reads it has first
+ * written itself, but two calls whose kernels overlap on the GPU (different streams, no
+ * ordering) race on it and give undefined results.  Asynchronous on `stream`. */
+int32_t dgc_decode_accumulate_static(int32_t num_workers, const int32_t* const* idx_lists,
+                                     const float* const* val_lists, const int64_t* nnz,
+                                     float* dense_out, int64_t dense_len, void* stream);
 
 /* Algorithm 4, line "theta <- SGD(theta, G_t)" with Eq. 5's third term:
  * w[i] <- w[i] - lr * dense_grad[i], two separately rounded fp32 operations.

@@ -59,6 +59,9 @@ _sigs = {
                                                ctypes.POINTER(_vp), _i64p, _vp, ctypes.c_int64,
                                                _vp, ctypes.c_int64, _vp]),
     "dgc_decode_workspace_bytes": (ctypes.c_int64, [ctypes.c_int32, ctypes.c_int64]),
+    "dgc_decode_accumulate_static": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
+                                                      ctypes.POINTER(_vp), _i64p, _vp,
+                                                      ctypes.c_int64, _vp]),
     "dgc_apply_sgd": (ctypes.c_int32, [_vp, _vp, ctypes.c_int64, ctypes.c_float, _vp]),
     "dgc_get_status": (ctypes.c_int32, [_vp, _vp, ctypes.POINTER(Status)]),
     "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
@@ -232,6 +235,26 @@ def decode_accumulate(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[tor
                                       dense_out.numel(), workspace.data_ptr(),
                                       workspace.numel() * workspace.element_size(),
                                       _stream(stream)), "dgc_decode_accumulate")
+
+
+STATIC_DECODE_WORDS = 1 << 18
+
+
+def decode_accumulate_static(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[torch.Tensor],
+                             dense_out: torch.Tensor, stream=None,
+                             nnz: Optional[Sequence[int]] = None) -> None:
+    """dgc_decode_accumulate without a workspace argument, for callers that may not allocate
+    device memory: the scratch is a fixed 1 MiB array inside the library.  Raises DgcError
+    (ECAPACITY) when workers x (tiles + 1) exceeds STATIC_DECODE_WORDS.  Calls on one device
+    share that scratch, so do not let two of them overlap on the GPU."""
+    n = len(idx_lists)
+    ip = (_vp * n)(*[_dev(t, torch.int32) for t in idx_lists])
+    vp = (_vp * n)(*[_dev(t, torch.float32) for t in val_lists])
+    cnt = (ctypes.c_int64 * n)(*[int(c) for c in (nnz if nnz is not None
+                                                  else [t.numel() for t in idx_lists])])
+    _check(_lib.dgc_decode_accumulate_static(n, ip, vp, cnt, _dev(dense_out, torch.float32),
+                                             dense_out.numel(), _stream(stream)),
+           "dgc_decode_accumulate_static")
 
 
 def apply_sgd(w: torch.Tensor, dense_grad: torch.Tensor, lr: float, stream=None) -> None:

@@ -629,3 +629,64 @@ int32_t dgc_state_write(dgc_state* st, const float* u_host, const float* v_host,
 }
 
 }  // extern "C"
+
+// ====================================================================== allocation-free decode
+// Scratch of dgc_decode_accumulate_static: the per-worker tile boundaries that the caller of
+// dgc_decode_accumulate passes as `workspace`.  It lives in the library image, so every GPU
+// that loads the library holds DGC_STATIC_DECODE_WORDS * 4 bytes of it until the process exits.
+// In host code this name is only a stand-in for the symbol, not a device address: the address
+// a kernel may use comes from cudaGetSymbolAddress, asked once per device (below).
+static __device__ __align__(256) int32_t g_static_decode_bounds[DGC_STATIC_DECODE_WORDS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::atomic<int32_t*> g_static_bounds_ptr[kMaxDevices];   // device address per ordinal, 0 = not asked yet
+}  // namespace
+
+extern "C" int32_t dgc_decode_accumulate_static(int32_t num_workers,
+                                                 const int32_t* const* idx_lists,
+                                                 const float* const* val_lists, const int64_t* nnz,
+                                                 float* dense_out, int64_t dense_len, void* stream) {
+  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
+  if (!idx_lists || !val_lists || !nnz || dense_len < 0 || dense_len >= (int64_t)1 << 31)
+    return DGC_EINVAL;
+  if (dense_len == 0) return DGC_OK;
+  if (!dense_out) return DGC_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(dense_out) & 15u) != 0) return DGC_EINVAL;
+  const int64_t tiles = (dense_len + kDecodeTile - 1) / kDecodeTile;
+  // the fixed scratch bounds the problem: workers x (tiles + 1) boundary words must fit
+  if ((int64_t)num_workers * (tiles + 1) > (int64_t)DGC_STATIC_DECODE_WORDS) return DGC_ECAPACITY;
+  DecodeArgs a{};
+  int64_t max_nnz = 0;
+  for (int w = 0; w < num_workers; ++w) {
+    if (nnz[w] < 0 || nnz[w] > dense_len) return DGC_EINVAL;
+    if (nnz[w] > 0 && (!idx_lists[w] || !val_lists[w])) return DGC_EINVAL;
+    a.idx[w] = idx_lists[w];
+    a.val[w] = val_lists[w];
+    a.nnz[w] = (int32_t)nnz[w];
+    max_nnz = std::max(max_nnz, nnz[w]);
+  }
+  a.num_workers = num_workers;
+  a.num_tiles = (int32_t)tiles;
+  // set-up, once per device, with that device current: the symbol's device address
+  int dev = -1;
+  DGC_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return DGC_EINVAL;
+  int32_t* bounds = g_static_bounds_ptr[dev].load(std::memory_order_acquire);
+  if (!bounds) {
+    void* sym = nullptr;
+    DGC_CUDA(cudaGetSymbolAddress(&sym, g_static_decode_bounds));
+    if (!sym) return DGC_ECUDA;
+    bounds = static_cast<int32_t*>(sym);
+    g_static_bounds_ptr[dev].store(bounds, std::memory_order_release);
+  }
+  // nothing needs clearing: k_decode_bounds writes every boundary word [0, tiles] of every worker
+  // before k_decode_tiles reads it, so the previous call's contents are never seen
+  cudaStream_t s = as_stream(stream);
+  int32_t rc;
+  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
+  k_decode_bounds<<<dim3(gx, num_workers), 256, 0, s>>>(a, bounds);
+  if ((rc = check_launch()) != DGC_OK) return rc;
+  k_decode_tiles<<<a.num_tiles, kDecodeThreads, 0, s>>>(a, bounds, dense_out, dense_len);
+  return check_launch();
+}
