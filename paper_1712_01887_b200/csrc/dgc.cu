@@ -266,7 +266,8 @@ int32_t upload_plan(dgc_state* st, bool first) {
   int keys = (int)std::min<int64_t>(st->max_tensor_expect, key_cap);
   keys = std::max(keys, 1024);
   st->select_smem_keys = keys;
-  DGC_CUDA(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize, keys * 4));
+  DGC_CUDA(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (keys + kHistWords(kSelectThreads)) * 4));
   return DGC_OK;
 }
 
@@ -449,7 +450,8 @@ int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, f
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (prof) DGC_CUDA(cudaEventRecord(ev[3], s));
-  k_select<<<p.num_tensors, kSelectThreads, (size_t)st->select_smem_keys * 4, s>>>(
+  k_select<<<p.num_tensors, kSelectThreads,
+             (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s>>>(
       p, st->select_smem_keys, parity);
   if ((rc = check_launch()) != DGC_OK) return rc;
   if (prof) DGC_CUDA(cudaEventRecord(ev[4], s));

@@ -40,12 +40,12 @@ namespace dgc {
 constexpr int kSeg = 512;              // elements per warp segment (4 x float4 per lane)
 constexpr int kPartSegs = 512;         // segments per part (256 Ki elements)
 constexpr int kSmallN = 8192;          // tensors up to this size are not sampled
-constexpr int kMaxSampleGroups = 8192; // float4 groups sampled per tensor at most
+constexpr int kMaxSampleGroups = 16384; // float4 groups sampled per tensor at most
 constexpr int kSampleThreads = 512;    // one sampled float4 group per thread and block
 constexpr int kSampleSurvivors = 4096;
 constexpr int kSelectThreads = 1024;
-constexpr int kSelectMaxSmemKeys = 53248;
-constexpr int kSelectMaxParts = 1024;  // parts of one tensor whose tables fit in shared memory
+constexpr int kSelectMaxSmemKeys = 51200;
+constexpr int kSelectMaxParts = 256;   // parts of one tensor whose tables fit in shared memory
 constexpr int kEmitThreads = kPartSegs;   // one thread per segment of the part
 constexpr int kEmitRegs = 8;              // candidates per thread kept in registers
 constexpr int kMaskStride = 17;           // words per segment in the winner bitmaps (16 + 1 pad)
@@ -171,44 +171,51 @@ __device__ __forceinline__ void block_excl_scan2(int a, int b, int* sh, int& ea,
 // number of times on every thread of the block (valid = false for padding
 // calls).  Every valid key lies in [base, maxkey]; only the bits in which
 // maxkey - base can differ are scanned, 8 per pass from the top.
-// hist: 512 words of shared memory (two 256-bin histograms, used alternately
-// so that one is cleared while the other is read), sh: 2 words.  The block
-// needs at least 288 threads.  Two barriers per pass plus one.
+// Histograms: up to 16 private 256-bin copies (padded to 257 words so that the
+// same bin of different copies falls in different banks), one per warp or pair
+// of warps, so that the integer atomics of different warps do not collide;
+// they are folded into one of two alternating 256-bin histograms, in which
+// warp 0 finds the digit.  hist: kHistWords(blockDim.x) words of shared
+// memory, sh: 2 words.  blockDim.x is a multiple of 256, at least 512.
 // Returns the key; n_gt = number of keys strictly greater.
-constexpr int kHistWords = 512;
+__host__ __device__ constexpr int kHistCopies(int threads) { return threads / 32 < 16 ? threads / 32 : 16; }
+__host__ __device__ constexpr int kHistWords(int threads) { return kHistCopies(threads) * 257 + 512; }
 
 template <class ForEach>
 __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank, uint32_t base,
                                                       uint32_t maxkey, uint32_t* hist, int* sh,
                                                       int& n_gt) {
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
+  const int copies = kHistCopies(nt);
+  uint32_t* mine = hist + ((tid >> 5) % copies) * 257;
+  uint32_t* folded = hist + copies * 257;
   const uint32_t span = maxkey - base;
   const int passes = span == 0 ? 0 : (32 - __clz(span) + 7) / 8;
   uint32_t prefix = 0, mask = 0;
   int remaining = rank;
-  if (tid < 256) hist[tid] = 0;
+  for (int i = tid; i < copies * 257 + 512; i += nt) hist[i] = 0;
   __syncthreads();
   int cur = 0;
   for (int shift = 8 * (passes - 1); shift >= 0; shift -= 8, cur ^= 1) {
-    uint32_t* h = hist + cur * 256;
     for_each([&](bool valid, uint32_t key) {
       key -= base;
-      uint32_t d = 0;
-      if (valid && (key & mask) == prefix) d = (key >> shift) & 255u; else valid = false;
-      // keys cluster on a few digits in the leading passes: lanes that share the digit of
-      // the first valid lane are added with one atomic, the others one by one
-      const unsigned vm = __ballot_sync(0xFFFFFFFFu, valid);
-      if (vm != 0) {
-        const uint32_t d0 = __shfl_sync(0xFFFFFFFFu, d, __ffs(vm) - 1);
-        const unsigned m0 = __ballot_sync(0xFFFFFFFFu, valid && d == d0);
-        if (valid) {
-          if (d != d0) atomicAdd(&h[d], 1u);
-          else if (lane == __ffs(m0) - 1) atomicAdd(&h[d], (uint32_t)__popc(m0));
-        }
-      }
+      if (valid && (key & mask) == prefix) atomicAdd(&mine[(key >> shift) & 255u], 1u);
     });
     __syncthreads();
+    {
+      // fold (and clear) the private copies: thread t takes bin t & 255 of a slice of them
+      const int bin = tid & 255, groups = nt >> 8, grp = tid >> 8;
+      const int c0 = grp * copies / groups, c1 = (grp + 1) * copies / groups;
+      uint32_t t = 0;
+      for (int c = c0; c < c1; ++c) {
+        t += hist[c * 257 + bin];
+        hist[c * 257 + bin] = 0;
+      }
+      if (t) atomicAdd(&folded[cur * 256 + bin], t);
+    }
+    __syncthreads();
     if (tid < 32) {
+      const uint32_t* h = folded + cur * 256;
       const int hi = 255 - 8 * lane;          // this lane covers bins hi, hi-1, .., hi-7
       uint32_t loc[8];
       uint32_t s = 0;
@@ -225,7 +232,7 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
         }
       }
     } else if (tid < 288) {
-      hist[(cur ^ 1) * 256 + tid - 32] = 0;   // clear the other histogram for the next pass
+      folded[(cur ^ 1) * 256 + tid - 32] = 0;   // clear the other histogram for the next pass
     }
     __syncthreads();
     prefix |= (uint32_t)sh[0] << shift;
@@ -322,7 +329,7 @@ k_sumsq(Plan p, const float* __restrict__ g, double thr_local, int clip_on) {
 template <bool CLIP>
 __global__ void __launch_bounds__(kSampleThreads)
 k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_seed) {
-  __shared__ uint32_t hist[kHistWords];
+  __shared__ uint32_t hist[kHistWords(kSampleThreads)];
   __shared__ uint32_t surv[kSampleSurvivors];
   __shared__ int sh[2];
   __shared__ int s_cnt;
@@ -559,8 +566,9 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
 // to the lower index, so to the earlier part).  One block per tensor.
 __global__ void __launch_bounds__(kSelectThreads)
 k_select(Plan p, int smem_keys, int parity) {
-  extern __shared__ uint32_t skeys[];
-  __shared__ uint32_t hist[kHistWords];
+  extern __shared__ uint32_t dyn_smem[];          // [histograms | keys]
+  uint32_t* hist = dyn_smem;
+  uint32_t* skeys = dyn_smem + kHistWords(kSelectThreads);
   __shared__ int sh[66];
   __shared__ int s_flag;
   __shared__ uint32_t s_max;
@@ -630,21 +638,23 @@ k_select(Plan p, int smem_keys, int parity) {
     return;
   }
   const bool in_smem = tables && total <= smem_keys;
+  const int slices = max(1, (kSelectThreads / 32) / pn);
   uint32_t kmax = 0x7FFFFFFFu;
   uint32_t kbase = 0u;
   if (in_smem) {
-    // gather the keys of all parts, compact, into shared memory: every load independent
+    // gather the keys of all parts, compact, into shared memory: coalesced reads, a part is
+    // shared by `slices` warps when the tensor has fewer parts than the block has warps
     uint32_t tmax = 0;
+    for (int unit = warp; unit < pn * slices; unit += kSelectThreads / 32) {
+      const int q = unit / slices, sl = unit - q * slices;
+      const int b0 = s_pbase[q], c = s_pbase[q + 1] - b0;
+      const float* src = p.cand_val + s_pcb[q];
 #pragma unroll 4
-    for (int i = tid; i < total; i += kSelectThreads) {
-      int lo = 0, hi = pn;                       // largest q with s_pbase[q] <= i
-      while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (s_pbase[mid] <= i) lo = mid; else hi = mid;
+      for (int i = sl * 32 + lane; i < c; i += slices * 32) {
+        const uint32_t key = mag_key(__ldcg(src + i));
+        skeys[b0 + i] = key;
+        tmax = max(tmax, key);
       }
-      const uint32_t key = mag_key(__ldcg(p.cand_val + s_pcb[lo] + (i - s_pbase[lo])));
-      skeys[i] = key;
-      tmax = max(tmax, key);
     }
     const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
     if (lane == 0) atomicMax(&s_max, wmax);
@@ -684,28 +694,30 @@ k_select(Plan p, int smem_keys, int parity) {
   const int quota = k - n_gt;   // ties (|v'| == kth) to take, lowest indices first
   const int out_off = t.out_off;
   if (tables) {
-    // per part: strictly-greater and tied candidates; one warp per part
-    for (int q = warp; q < pn; q += kSelectThreads / 32) {
-      int gt = 0, eq = 0;
-      if (in_smem) {
-        const int b0 = s_pbase[q], b1 = s_pbase[q + 1];
-        for (int i = b0 + lane; i < b1; i += 32) {
-          const uint32_t key = skeys[i];
+    // per part: strictly-greater and tied candidates (a single part needs no count: it takes
+    // the whole quota and k_emit_mask stops at the quota by itself)
+    for (int q = tid; q < pn; q += kSelectThreads) { s_gt[q] = 0; s_eq[q] = 0; }
+    __syncthreads();
+    if (pn > 1) {
+      for (int unit = warp; unit < pn * slices; unit += kSelectThreads / 32) {
+        const int q = unit / slices, sl = unit - q * slices;
+        const int b0 = s_pbase[q], c = s_pbase[q + 1] - b0;
+        const float* src = p.cand_val + s_pcb[q];
+        int gt = 0, eq = 0;
+        for (int i = sl * 32 + lane; i < c; i += slices * 32) {
+          const uint32_t key = in_smem ? skeys[b0 + i] : mag_key(__ldcg(src + i));
           gt += key > kth;
           eq += key == kth;
         }
-      } else {
-        const int c = s_pbase[q + 1] - s_pbase[q];
-        const float* src = p.cand_val + s_pcb[q];
-        for (int i = lane; i < c; i += 32) {
-          const uint32_t key = mag_key(__ldcg(src + i));
-          gt += key > kth;
-          eq += key == kth;
+        gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+        eq = __reduce_add_sync(0xFFFFFFFFu, eq);
+        if (lane == 0) {
+          if (gt) atomicAdd(&s_gt[q], gt);
+          if (eq) atomicAdd(&s_eq[q], eq);
         }
       }
-      gt = __reduce_add_sync(0xFFFFFFFFu, gt);
-      eq = __reduce_add_sync(0xFFFFFFFFu, eq);
-      if (lane == 0) { s_gt[q] = gt; s_eq[q] = eq; }
+    } else if (tid == 0) {
+      s_eq[0] = quota;     // upper bound is enough for one part
     }
     __syncthreads();
     if (pn <= 32) {
@@ -856,7 +868,7 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   __shared__ int sh[66];
   __shared__ int s_gtb[kPartSegs];             // winners before each segment
   __shared__ int s_eqb[kPartSegs];
-  static_assert(kEmitSmemBytes >= kHistWords * 4, "bitmaps double as histograms");
+  static_assert(kEmitSmemBytes >= kHistWords(kEmitThreads) * 4, "bitmaps double as histograms");
   uint32_t* mgt = smask;
   uint32_t* meq = smask + kPartSegs * kMaskStride;
   const int part = blockIdx.x;
