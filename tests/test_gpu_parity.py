@@ -78,6 +78,36 @@ def test_deepspeech_small_warmup_schedule(P):
     _run_workload(P, wl, 10, workers=2, schedule=lambda t: stages[min(t // 2, 4)])
 
 
+def test_lstm_full_size_one_worker(P):
+    """The 66,034,000-value LSTM-shaped set at full size (15 M-element tensors, 58 parts each):
+    every index, value and state word against the oracle, clipping on."""
+    wl = I.workload("lstm")
+    rep = _run_workload(P, wl, 2, workers=1, receive=False)
+    assert rep.full_select == 0
+
+
+def test_deepspeech_full_size_two_warmup_stages(P):
+    """The 122,096,829-value DeepSpeech-shaped set at full size: one iteration at 75 % and
+    one at 99.9 % sparsity (k = 30.5 M and 122 K entries)."""
+    wl = I.workload("deepspeech")
+    stages = [0.75, 0.999]
+    _run_workload(P, wl, 2, workers=1, receive=False, schedule=lambda t: stages[t])
+
+
+@pytest.mark.parametrize("n", [1 << 16, 1 << 18, 1 << 20, 1 << 22, 1 << 24])
+@pytest.mark.parametrize("sparsity", [0.99, 0.999, 0.9999])
+def test_sweep_single_tensor(P, n, sparsity):
+    wl = I.workload("sweep", n=n, sparsity=sparsity)
+    rep = _run_workload(P, wl, 2, workers=1)
+    assert rep.full_select == 0
+
+
+@pytest.mark.parametrize("n,sparsity", [(1 << 26, 0.999), (1 << 28, 0.999), (1 << 28, 0.99)])
+def test_sweep_largest_tensors(P, n, sparsity):
+    wl = I.workload("sweep", n=n, sparsity=sparsity)
+    _run_workload(P, wl, 1 if n == 1 << 28 else 2, workers=1, receive=False)
+
+
 @pytest.mark.parametrize("sparsity", [0.999, 0.99, 0.75, 0.0])
 def test_edge_sizes(P, sparsity):
     numel = [1, 3, 4, 5, 31, 32, 33, 511, 512, 513, 4095, 4096, 4097, 8192, 8193, 70001,
