@@ -65,6 +65,7 @@ struct dgc_state {
   std::vector<int32_t> seg_part;
   std::vector<SampleBlock> sample_blocks;
   int64_t sample_keys_total = 0;
+  std::vector<int32_t> big_parts, big_tensors;   // multi-block selection path
   int64_t max_nnz = 0;
   int64_t cand_total = 0;
   int64_t max_tensor_expect = 0;   // largest expected candidate count of one tensor
@@ -115,6 +116,12 @@ void dev_free(dgc_state* st, void* ptr) {
 
 // Everything that depends on the sparsity: k, output offsets, sampling plan,
 // candidate capacities.  Segments and parts depend only on the shapes.
+// Keys one k_select block may hold in shared memory: two blocks per SM when there are more
+// tensors than SMs, else one large block.
+int select_key_cap(const dgc_state* st) {
+  return st->cfg.num_tensors > st->sm_count ? 16384 : kSelectMaxSmemKeys;
+}
+
 void build_host_plan(dgc_state* st, double sparsity) {
   const int T = st->cfg.num_tensors;
   const double ratio = st->cfg.sample_ratio > 0.0 ? st->cfg.sample_ratio : 0.01;
@@ -123,6 +130,9 @@ void build_host_plan(dgc_state* st, double sparsity) {
   st->seg_part.clear();
   st->sample_blocks.clear();
   st->sample_keys_total = 0;
+  st->big_parts.clear();
+  st->big_tensors.clear();
+  const int key_cap = select_key_cap(st);
   int64_t pos = 0, out = 0, cbase = 0;
   st->max_tensor_expect = 0;
   for (int j = 0; j < T; ++j) {
@@ -144,6 +154,10 @@ void build_host_plan(dgc_state* st, double sparsity) {
     if (sampled) {
       const int64_t Q = n / 4;
       int64_t G = (int64_t)std::ceil(ratio * (double)n / 4.0);
+      // a sample that holds about 1024 of the entries to send pins the proposal to +-20 %;
+      // at low sparsity that needs far fewer than ratio * n elements
+      const int64_t enough = (int64_t)std::ceil(1024.0 / std::max(1.0 - sparsity, 1e-9) / 4.0);
+      G = std::min<int64_t>(G, enough);
       G = std::max<int64_t>(G, 64);
       G = std::min<int64_t>(G, std::min<int64_t>(Q, kMaxSampleGroups));
       const double S = 4.0 * (double)G;
@@ -169,6 +183,11 @@ void build_host_plan(dgc_state* st, double sparsity) {
     }
     t.part_first = (int32_t)st->pm.size();
     t.part_num = (int32_t)nparts;
+    // too many candidates (or parts) for one block: the multi-block selection path
+    const bool big = expect_keys > (double)key_cap || nparts > kSelectMaxParts;
+    t.big = big ? 1 : 0;
+    t.big_slot = big ? (int32_t)st->big_tensors.size() : -1;
+    if (big) st->big_tensors.push_back(j);
     for (int64_t q = 0; q < nparts; ++q) {
       const int64_t seg0 = pos / kSeg + q * kPartSegs;
       const int64_t ns = std::min<int64_t>(kPartSegs, nseg - q * kPartSegs);
@@ -187,11 +206,13 @@ void build_host_plan(dgc_state* st, double sparsity) {
       m.cbase = (int32_t)cbase;
       m.cap = (int32_t)cap;
       m.first = q == 0 ? 1 : 0;
+      m.big_slot = big ? (int32_t)st->big_parts.size() : -1;
+      if (big) st->big_parts.push_back((int32_t)st->pm.size());
       st->pm.push_back(m);
       cbase += cap;
       for (int64_t s = 0; s < ns; ++s) st->seg_part.push_back((int32_t)(st->pm.size() - 1));
     }
-    st->max_tensor_expect = std::max<int64_t>(st->max_tensor_expect, (int64_t)expect_keys);
+    if (!big) st->max_tensor_expect = std::max<int64_t>(st->max_tensor_expect, (int64_t)expect_keys);
     pos += nseg * kSeg;
   }
   st->arena_len = pos;
@@ -218,6 +239,13 @@ int32_t upload_plan(dgc_state* st, bool first) {
   const size_t o_samp = o; o = up16(o + NS * sizeof(SampleBlock));
   const size_t o_skeys = o; o = up16(o + (size_t)st->sample_keys_total * 4);
   const size_t o_stick = o; o = up16(o + T * 4);
+  const size_t NBP = st->big_parts.size(), NBT = st->big_tensors.size();
+  const size_t o_bparts = o; o = up16(o + NBP * 4);
+  const size_t o_btens = o; o = up16(o + NBT * 4);
+  const size_t o_bhist = o; o = up16(o + NBT * 3 * kBigBins * 4);
+  const size_t o_bstate = o; o = up16(o + NBT * kBigStateWords * 4);
+  const size_t o_babove = o; o = up16(o + NBP * 4);
+  const size_t o_blast = o; o = up16(o + NBP * kBigLastStride * 4);
   const size_t bytes = o + 16;
   if (first || bytes > st->d_tables_bytes) {
     if (st->d_tables) dev_free(st, st->d_tables);
@@ -232,6 +260,8 @@ int32_t upload_plan(dgc_state* st, bool first) {
   std::memcpy(h.data() + o_pm, st->pm.data(), P * sizeof(PartMeta));
   std::memcpy(h.data() + o_seg, st->seg_part.data(), S * 4);
   if (NS) std::memcpy(h.data() + o_samp, st->sample_blocks.data(), NS * sizeof(SampleBlock));
+  if (NBP) std::memcpy(h.data() + o_bparts, st->big_parts.data(), NBP * 4);
+  if (NBT) std::memcpy(h.data() + o_btens, st->big_tensors.data(), NBT * 4);
   DGC_CUDA(cudaMemcpy(st->d_tables, h.data(), bytes, cudaMemcpyHostToDevice));
   char* d = st->d_tables;
   Plan& p = st->plan;
@@ -246,6 +276,13 @@ int32_t upload_plan(dgc_state* st, bool first) {
   p.sample_blocks = (const SampleBlock*)(d + o_samp);
   p.sample_keys = (uint32_t*)(d + o_skeys);
   p.sample_ticket = (int32_t*)(d + o_stick);
+  p.big_parts = (const int32_t*)(d + o_bparts);
+  p.big_tensors = (const int32_t*)(d + o_btens);
+  p.big_hist = (int32_t*)(d + o_bhist);
+  p.big_state = (int32_t*)(d + o_bstate);
+  p.big_above = (int32_t*)(d + o_babove);
+  p.big_last = (int32_t*)(d + o_blast);
+  p.num_big_parts = (int32_t)NBP; p.num_big_tensors = (int32_t)NBT;
   p.num_tensors = (int32_t)T; p.num_parts = (int32_t)P; p.num_segs = (int32_t)S;
   // candidate lists
   if (st->cand_total > st->cand_alloc) {
@@ -261,9 +298,7 @@ int32_t upload_plan(dgc_state* st, bool first) {
   }
   p.cand_idx = st->d_cand_idx; p.cand_val = st->d_cand_val;
   // shared memory of the select kernel
-  // two select blocks per SM when there are more tensors than SMs, else one big one
-  const int key_cap = st->cfg.num_tensors > st->sm_count ? 16384 : kSelectMaxSmemKeys;
-  int keys = (int)std::min<int64_t>(st->max_tensor_expect, key_cap);
+  int keys = (int)std::min<int64_t>(st->max_tensor_expect, select_key_cap(st));
   keys = std::max(keys, 1024);
   st->select_smem_keys = keys;
   DGC_CUDA(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -454,6 +489,16 @@ int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, f
              (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s>>>(
       p, st->select_smem_keys, parity);
   if ((rc = check_launch()) != DGC_OK) return rc;
+  if (p.num_big_parts > 0) {
+    k_big_hist<0><<<p.num_big_parts, kBigThreads, 0, s>>>(p);
+    if ((rc = check_launch()) != DGC_OK) return rc;
+    k_big_hist<1><<<p.num_big_parts, kBigThreads, 0, s>>>(p);
+    if ((rc = check_launch()) != DGC_OK) return rc;
+    k_big_hist<2><<<p.num_big_parts, kBigThreads, 0, s>>>(p);
+    if ((rc = check_launch()) != DGC_OK) return rc;
+    k_big_final<<<p.num_big_tensors, kSelectThreads, 0, s>>>(p, parity);
+    if ((rc = check_launch()) != DGC_OK) return rc;
+  }
   if (prof) DGC_CUDA(cudaEventRecord(ev[4], s));
   k_emit_mask<<<p.num_parts, kEmitThreads, kEmitSmemBytes, s>>>(p, out_idx, out_val);
   if ((rc = check_launch()) != DGC_OK) return rc;

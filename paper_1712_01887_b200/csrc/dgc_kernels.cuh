@@ -53,6 +53,12 @@ constexpr int kEmitSmemBytes = 2 * kPartSegs * kMaskStride * 4;
 constexpr int kMainThreads = 256;
 constexpr int kNormThreads = 256;
 constexpr int kMaxNormGrid = 2048;
+constexpr int kBigThreads = 512;
+constexpr int kBigBins = 2048;         // 11-bit digits: key bits 30..20, 19..9, then 9 bits 8..0
+constexpr int kBigLastBins = 512;
+constexpr int kBigLastStride = 516;    // 513 suffix sums, padded to a multiple of 4 words
+constexpr int kBigStateWords = 64;
+constexpr int kBigNear = 64;           // round-0 digits this close above the proposal's get private bins
 constexpr int kDecodeTile = 4096;
 constexpr int kDecodeThreads = 256;
 
@@ -63,14 +69,14 @@ struct __align__(16) TensorMeta {   // one per tensor, read-only for the kernels
   int32_t part_first, part_num;
   int32_t rank, groups;             // sampling: rank of the proposal, float4 groups sampled
   int32_t key_base, chunks;         // sampling: first key in the sample buffer, blocks that sample
-  int32_t pad0, pad1;
+  int32_t big, big_slot;            // big: selected by the multi-block path; slot in its tables
 };
 struct SampleBlock { int32_t tensor, chunk; };   // work item of one k_sample_threshold block
 struct __align__(16) PartMeta {     // one per part (up to kPartSegs segments of one tensor)
   int32_t tensor, end;              // end: arena index one past the part's last real element
   int32_t seg0, nseg;
   int32_t cbase, cap;               // candidate list of the part
-  int32_t first, pad;               // first: this is the tensor's first part
+  int32_t first, big_slot;          // first: the tensor's first part; slot among the big parts or -1
 };
 struct __align__(16) PartSel {      // written by k_select, read by k_emit_mask
   uint32_t kth;                     // bit pattern of the k-th largest |v'| of the tensor
@@ -91,6 +97,15 @@ struct Plan {
   const SampleBlock* sample_blocks;
   uint32_t* sample_keys;     // |v'| keys of the current call's sample, all tensors
   int32_t* sample_ticket;    // per tensor: sampling blocks that have finished
+  // multi-block selection (tensors with too many candidates for one block)
+  const int32_t* big_parts;  // parts of the big tensors
+  const int32_t* big_tensors;
+  int32_t* big_hist;         // [big tensor][3][2048] digit histograms of the three rounds
+  int32_t* big_state;        // [big tensor][64]: prefix and remaining rank after round 0 (words
+                             // 0,1) and after round 1 (words 32,33: a cache line of their own)
+  int32_t* big_above;        // [big part]: candidates whose upper 22 key bits exceed the prefix
+  int32_t* big_last;         // [big part][513]: suffix sums of the part's last-round digit
+                             // counts: word d = candidates matching the prefix with digit >= d
   int32_t* cand_idx;
   float* cand_val;
   float* coef;
@@ -101,6 +116,7 @@ struct Plan {
   float* u;
   float* v;
   int32_t num_tensors, num_parts, num_segs;
+  int32_t num_big_parts, num_big_tensors;
 };
 
 template <class T>
@@ -582,6 +598,7 @@ k_select(Plan p, int smem_keys, int parity) {
   const int p0 = t.part_first, pn = t.part_num, k = t.k;
   const bool tables = pn <= kSelectMaxParts;
   if (j == 0 && tid < 4) p.diag[(parity ^ 1) * 4 + tid] = 0;   // next call's counters
+  if (t.big) return;                                            // k_big_* select this tensor
   if (tid == 0) { s_flag = 0; s_max = 0u; }
   __syncthreads();
   // candidates per part (one load round for all parts), overflow check, compact bases
@@ -794,6 +811,232 @@ k_select(Plan p, int smem_keys, int parity) {
   }
 }
 
+// ------------------------------------------------------------------ K4b: multi-block exact k-th key
+// The same selection for tensors whose candidates do not fit one block's shared
+// memory (warm-up sparsities, very large tensors): a radix select over the 31
+// key bits in three rounds (11 + 11 + 9 bits), one block per part and round.
+// Each round adds the part's digit counts to the tensor's histogram in global
+// memory (integer atomics); the next round's blocks each read that histogram,
+// find the digit that holds the k-th key (all blocks of a tensor compute the
+// same value) and count the next digit among the keys that match the prefix.
+// k_big_final then derives the threshold, every part's share and output base.
+// No block waits for another: rounds are separate launches.
+
+// The digit (counting from the largest) at which the cumulative count reaches
+// `remaining`; returns the digit, `above` = keys in larger digits.  All threads
+// of the block get the result.  bins <= 4 * blockDim.x.  sh: 66 + 2 ints.
+__device__ __forceinline__ int block_find_digit(const int32_t* hist, int bins, int remaining,
+                                                int* sh, int& above) {
+  const int tid = threadIdx.x;
+  const int per = (bins + blockDim.x - 1) / blockDim.x;      // bins per thread, descending order
+  int loc[4];
+  int sum = 0;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const int bin = bins - 1 - (tid * per + q);
+    loc[q] = (q < per && bin >= 0) ? __ldcg(hist + bin) : 0;
+    sum += loc[q];
+  }
+  int ex, dummy, tot, dummy2;
+  block_excl_scan2(sum, 0, sh, ex, dummy, tot, dummy2);
+  if (ex < remaining && remaining <= ex + sum) {
+    int c = ex;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (c + loc[q] >= remaining) { sh[66] = bins - 1 - (tid * per + q); sh[67] = c; break; }
+      c += loc[q];
+    }
+  }
+  __syncthreads();
+  const int digit = sh[66];
+  above = sh[67];
+  __syncthreads();
+  return digit;
+}
+
+template <int ROUND>
+__global__ void __launch_bounds__(kBigThreads)
+k_big_hist(Plan p) {
+  __shared__ int hist[kBigBins];
+  __shared__ int near[(kBigThreads / 32) * kBigNear];   // round 0: private bins near the proposal
+  __shared__ int sh[68];
+  __shared__ int s_above;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int part = __ldg(p.big_parts + blockIdx.x);
+  const PartMeta pm = load_record(p.pm + part);
+  const TensorMeta t = load_record(p.tm + pm.tensor);
+  const int count = min(__ldcg(p.p_count + part), pm.cap);
+  int32_t* thist = p.big_hist + (size_t)t.big_slot * 3 * kBigBins;
+  int32_t* state = p.big_state + t.big_slot * kBigStateWords;
+  // the prefix fixed by the earlier rounds
+  uint32_t prefix = 0;        // upper key bits already decided (11 after round 0, 22 after round 1)
+  if (ROUND == 1) {
+    int above;
+    const int d0 = block_find_digit(thist, kBigBins, t.k, sh, above);
+    prefix = (uint32_t)d0;
+    // every block of the tensor computes the same values; its first part's block records them
+    if (tid == 0 && pm.first) { state[0] = d0; state[1] = t.k - above; }
+  } else if (ROUND == 2) {
+    const int d0 = __ldcg(state + 0), rem1 = __ldcg(state + 1);
+    int above;
+    const int d1 = block_find_digit(thist + kBigBins, kBigBins, rem1, sh, above);
+    prefix = ((uint32_t)d0 << 11) | (uint32_t)d1;
+    if (tid == 0 && pm.first) { state[32] = (int)prefix; state[33] = rem1 - above; }
+  }
+  for (int i = tid; i < kBigBins; i += kBigThreads) hist[i] = 0;
+  if (ROUND == 0) for (int i = tid; i < (kBigThreads / 32) * kBigNear; i += kBigThreads) near[i] = 0;
+  if (tid == 0) s_above = 0;
+  __syncthreads();
+  const float* cval = p.cand_val + pm.cbase;
+  const int dthr = (int)(__ldcg(p.p_thr + part) >> 20);     // round-0 digit of the proposal
+  int above_cnt = 0;
+  for (int i0 = 0; i0 < count; i0 += kBigThreads * 4) {
+    float vals[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = i0 + b * kBigThreads + tid;
+      vals[b] = i < count ? __ldcg(cval + i) : 0.0f;
+    }
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = i0 + b * kBigThreads + tid;
+      if (i < count) {
+        const uint32_t key = mag_key(vals[b]);
+        if (ROUND == 0) {
+          // candidates crowd into the few digits just above the proposal: those go to a
+          // per-warp private histogram, the rest to the shared one
+          const int d = (int)(key >> 20), rel = d - dthr;
+          if (rel >= 0 && rel < kBigNear) atomicAdd(&near[warp * kBigNear + rel], 1);
+          else atomicAdd(&hist[d], 1);
+        } else if (ROUND == 1) {
+          if ((key >> 20) == prefix) atomicAdd(&hist[(key >> 9) & 2047u], 1);
+        } else {
+          const uint32_t up = key >> 9;
+          if (up == prefix) atomicAdd(&hist[key & 511u], 1);
+          else if (up > prefix) ++above_cnt;
+        }
+      }
+    }
+  }
+  if (ROUND == 2) {
+    above_cnt = __reduce_add_sync(0xFFFFFFFFu, above_cnt);
+    if (lane == 0 && above_cnt) atomicAdd(&s_above, above_cnt);
+  }
+  __syncthreads();
+  if (ROUND == 0) {
+    for (int r = tid; r < kBigNear; r += kBigThreads) {
+      int c = 0;
+      for (int w = 0; w < kBigThreads / 32; ++w) c += near[w * kBigNear + r];
+      if (c && dthr + r < kBigBins) atomicAdd(&hist[dthr + r], c);
+    }
+    __syncthreads();
+  }
+  int32_t* ghist = thist + ROUND * kBigBins;
+  const int bins = ROUND == 2 ? kBigLastBins : kBigBins;
+  for (int i = tid; i < bins; i += kBigThreads) {
+    const int c = hist[i];
+    if (c) atomicAdd(ghist + i, c);
+  }
+  if (ROUND == 2) {
+    // what k_big_final needs of this part: for every digit d, the candidates that match the
+    // prefix with last digit >= d (thread t holds digit 511 - t so that the scan runs downwards)
+    static_assert(kBigThreads == kBigLastBins, "one last-round bin per thread");
+    const int c = hist[kBigLastBins - 1 - tid];
+    int ex, dummy, tot, dummy2;
+    block_excl_scan2(c, 0, sh, ex, dummy, tot, dummy2);
+    int32_t* L = p.big_last + (size_t)pm.big_slot * kBigLastStride;
+    L[kBigLastBins - 1 - tid] = ex + c;
+    if (tid == 0) { L[kBigLastBins] = 0; p.big_above[pm.big_slot] = s_above; }
+  }
+}
+
+__global__ void __launch_bounds__(kSelectThreads)
+k_big_final(Plan p, int parity) {
+  __shared__ int sh[68];
+  __shared__ int s_gt[kSelectThreads];
+  __shared__ int s_eq[kSelectThreads];
+  const int tid = threadIdx.x;
+  const int j = __ldg(p.big_tensors + blockIdx.x);
+  const TensorMeta t = load_record(p.tm + j);
+  const int p0 = t.part_first, pn = t.part_num, k = t.k;
+  int32_t* thist = p.big_hist + (size_t)t.big_slot * 3 * kBigBins;
+  const int32_t* state = p.big_state + t.big_slot * kBigStateWords;
+  // total candidates and overflow
+  int mine = 0, over = 0;
+  for (int q = tid; q < pn; q += kSelectThreads) {
+    const int c = __ldcg(p.p_count + p0 + q);
+    const int cap = __ldg(&p.pm[p0 + q].cap);
+    over |= c > cap;
+    mine += min(c, cap);
+  }
+  int ex, exo, total, overflow;
+  block_excl_scan2(mine, over, sh, ex, exo, total, overflow);
+  __syncthreads();
+  const bool dense = overflow != 0 || total < k;
+  uint32_t kth = 0;
+  int quota = 0;
+  if (!dense) {
+    const uint32_t prefix = (uint32_t)__ldcg(state + 32);
+    const int rem2 = __ldcg(state + 33);
+    int above;
+    const int d2 = block_find_digit(thist + 2 * kBigBins, kBigLastBins, rem2, sh, above);
+    kth = (prefix << 9) | (uint32_t)d2;
+    quota = rem2 - above;                       // ties with kth to send, lowest indices first
+    // parts in chunks of blockDim: one warp per part reads its last-round counts
+    int run_gt = 0, run_eq = 0;
+    for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+      s_gt[tid] = 0;
+      s_eq[tid] = 0;
+      const int qn = min(kSelectThreads, pn - q0);
+      if (tid < qn) {
+        const int slot = __ldg(&p.pm[p0 + q0 + tid].big_slot);
+        const int32_t* L = p.big_last + (size_t)slot * kBigLastStride;
+        const int ge = __ldcg(L + d2), gtl = __ldcg(L + d2 + 1);
+        s_gt[tid] = gtl + __ldcg(p.big_above + slot);
+        s_eq[tid] = ge - gtl;
+      }
+      __syncthreads();
+      const int gt = s_gt[tid], eq = s_eq[tid];
+      int bg, be, tg, te;
+      block_excl_scan2(gt, eq, sh, bg, be, tg, te);
+      bg += run_gt;
+      be += run_eq;
+      if (tid < qn) {
+        PartSel ps;
+        ps.kth = kth;
+        ps.quota = max(0, min(quota - be, eq));
+        ps.out_base = t.out_off + bg + min(be, quota);
+        ps.dense = 0;
+        p.psel[p0 + q0 + tid] = ps;
+      }
+      run_gt += tg;
+      run_eq += te;
+      __syncthreads();
+    }
+  } else {
+    for (int q = tid; q < pn; q += kSelectThreads) {
+      PartSel ps;
+      ps.kth = 0u; ps.quota = 0; ps.out_base = 0; ps.dense = 1;
+      p.psel[p0 + q] = ps;
+    }
+  }
+  // histograms back to zero for the next call
+  for (int i = tid; i < 3 * kBigBins; i += kSelectThreads) thist[i] = 0;
+  if (tid == 0) {
+    if (dense) {
+      p.t_cand[j] = -1;
+      atomicOr((unsigned long long*)&p.diag[parity * 4 + 0],
+               (unsigned long long)(DGC_FLAG_FULL_SELECT |
+                                    (overflow ? DGC_FLAG_CAND_OVERFLOW : DGC_FLAG_CAND_SHORT)));
+      atomicAdd((unsigned long long*)&p.diag[parity * 4 + 1], 1ull);
+    } else {
+      p.t_kth[j] = kth;
+      p.t_cand[j] = total;
+      atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
+    }
+  }
+}
+
 // ------------------------------------------------------------------ K5: ordered emission + masking
 // Algorithm 4: G~[j] <- V[j] (.) Mask ; V[j] <- V[j] (.) !Mask ; U[j] <- U[j] (.) !Mask.
 // One block per part.  The candidates that reach the threshold set one bit
@@ -914,12 +1157,25 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
       atomicOr((key > kth ? mgt : meq) + word, 1u << (local & 31));
     }
   }
-  for (int i = kEmitRegs * kEmitThreads + tid; i < count; i += kEmitThreads) {
-    const uint32_t key = mag_key(__ldcg(cval + i));
-    if (key >= kth) {
-      const int local = __ldcg(cidx + i) - pm.seg0 * kSeg;
-      const int word = (local >> 9) * kMaskStride + ((local >> 5) & 15);
-      atomicOr((key > kth ? mgt : meq) + word, 1u << (local & 31));
+  // longer lists (low sparsity): the rest in batches of four loads per array
+  for (int i0 = kEmitRegs * kEmitThreads; i0 < count; i0 += 4 * kEmitThreads) {
+    float v4[4];
+    int x4[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = i0 + b * kEmitThreads + tid;
+      v4[b] = i < count ? __ldcg(cval + i) : 0.0f;
+      x4[b] = i < count ? __ldcg(cidx + i) : 0;
+    }
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = i0 + b * kEmitThreads + tid;
+      const uint32_t key = mag_key(v4[b]);
+      if (i < count && key >= kth) {
+        const int local = x4[b] - pm.seg0 * kSeg;
+        const int word = (local >> 9) * kMaskStride + ((local >> 5) & 15);
+        atomicOr((key > kth ? mgt : meq) + word, 1u << (local & 31));
+      }
     }
   }
   __syncthreads();
@@ -965,10 +1221,21 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
 #pragma unroll
   for (int b = 0; b < kEmitRegs; ++b)
     if (locs[b] >= 0) emit(locs[b], vals[b], mag_key(vals[b]));
-  for (int i = kEmitRegs * kEmitThreads + tid; i < count; i += kEmitThreads) {
-    const float val = __ldcg(cval + i);
-    const uint32_t key = mag_key(val);
-    if (key >= kth) emit(__ldcg(cidx + i) - pm.seg0 * kSeg, val, key);
+  for (int i0 = kEmitRegs * kEmitThreads; i0 < count; i0 += 4 * kEmitThreads) {
+    float v4[4];
+    int x4[4];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = i0 + b * kEmitThreads + tid;
+      v4[b] = i < count ? __ldcg(cval + i) : 0.0f;
+      x4[b] = i < count ? __ldcg(cidx + i) : 0;
+    }
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int i = i0 + b * kEmitThreads + tid;
+      const uint32_t key = mag_key(v4[b]);
+      if (i < count && key >= kth) emit(x4[b] - pm.seg0 * kSeg, v4[b], key);
+    }
   }
 }
 
