@@ -254,6 +254,26 @@ def run_ours(args):
     torch.cuda.synchronize()
     compress_ms = c0.elapsed_time(c1) / (K * NW)
 
+    # receive side alone: dense decode + SGD (what the step runs) and the fused sparse form
+    def _time(fn, reps=20):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        fn()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    def _dense_receive():
+        B.decode_accumulate(out_i, out_v, dense, ws)
+        B.apply_sgd(weights, dense, LR)
+
+    receive = {"decode_plus_sgd_ms": _time(_dense_receive),
+               "fused_sparse_decode_sgd_ms": _time(
+                   lambda: B.decode_apply_sgd(out_i, out_v, weights, LR, ws))}
+
     # end to end through the host-buffer entry point: H2D of every gradient and D2H of the
     # sparse lists inside the timed region
     e2e = None
@@ -322,7 +342,7 @@ def run_ours(args):
         "compress": {"ms_per_worker": compress_ms, "elements_per_s": total / (compress_ms * 1e-3),
                      "algorithmic_gbs": compress_bytes / (compress_ms * 1e-3) / 1e9,
                      "frac_of_peak": compress_bytes / (compress_ms * 1e-3) / 1e9 / peak},
-        "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
+        "receive": receive, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
     }
     print(json.dumps(line))
     if world > 1:

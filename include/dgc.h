@@ -66,6 +66,9 @@ typedef struct dgc_config {
   int32_t        debug_sample_rank; /* test hook: when > 0, the sampled threshold is taken at
                                      this rank of the sample instead of the safe one (rank 1 =
                                      sample maximum, which forces the full-selection path)     */
+  int32_t        nesterov;        /* 0: Algorithm 4 (vanilla momentum, Eq. 5).  1: Algorithm 5
+                                     (Appendix B): U <- m*(U + g) ; V <- (V + U) + g           */
+  int32_t        reserved;        /* set to 0                                                   */
 } dgc_config;
 
 typedef struct dgc_status {
@@ -114,7 +117,8 @@ int32_t dgc_layout(const dgc_state* st, int64_t* arena_offset, int64_t* k, int64
 /* One iteration of Algorithm 4 on this worker, from the clipping line to the
  * end of the loop over tensors (Sec. 3.2, Eq. 5, Sec. 3.3, Sec. 5):
  *   coef = min(1, thr_G N^-1/2 / ||g||_2) over the whole set (fp64 sum), gc = g*coef
- *   u <- m*u + gc ; v <- v + u            (separately rounded fp32 operations)
+ *   u <- m*u + gc ; v <- v + u            (separately rounded fp32 operations; with
+ *                                          cfg.nesterov: u <- m*(u + gc) ; v <- (v + u) + gc)
  *   per tensor j: the k_j entries of v largest in |v| (ties: lower index first)
  *   out: their (arena index, v) pairs, ascending index, at out_offset[j]
  *   v <- 0, u <- 0 at those entries (momentum factor masking)
@@ -186,6 +190,17 @@ int32_t dgc_decode_accumulate_static(int32_t num_workers, const int32_t* const* 
  * w[i] <- w[i] - lr * dense_grad[i], two separately rounded fp32 operations.
  * w and dense_grad are device arrays of len floats.  Asynchronous. */
 int32_t dgc_apply_sgd(float* w, const float* dense_grad, int64_t len, float lr, void* stream);
+
+/* Eq. 5, third term, applied directly: w <- w - lr * sum_k sparse(v_k) without forming
+ * the dense gradient.  Only the entries of w that some worker lists change; the result is
+ * bit for bit that of dgc_decode_accumulate followed by dgc_apply_sgd (the listed values are
+ * summed in worker order from +0, then w[i] <- w[i] - lr * G[i]; elsewhere w - lr * (+0) = w).
+ * Arguments as for dgc_decode_accumulate, with the weight array (device, len floats, read
+ * and written) in place of dense_out and the same workspace size.  Asynchronous. */
+int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_lists,
+                             const float* const* val_lists, const int64_t* nnz, float* w,
+                             int64_t len, float lr, void* workspace, int64_t workspace_bytes,
+                             void* stream);
 
 /* Synchronises `stream`, then reports counters of the last dgc_compress. */
 int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out);

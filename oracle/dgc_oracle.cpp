@@ -9,7 +9,8 @@
 // Steps and the passages they follow (Algorithm 4 = "Deep Gradient Compression
 // for vanilla momentum SGD on node k", Appendix D):
 //   clip coefficient        Sec. 3.2 "Local Gradient Clipping", Appendix C (thr * N^-1/2)
-//   momentum correction     Eq. 5 (u <- m u + g ; v <- v + u), Algorithm 4 lines "U <- ...", "V <- ..."
+//   momentum correction     Eq. 5 (u <- m u + g ; v <- v + u), Algorithm 4 lines "U <- ...", "V <- ...";
+//                           Nesterov form: Algorithm 5 / Appendix B Eq. 8
 //   per-tensor selection    Algorithm 4 inner loop over j (thr <- s% of |V[j]|, Mask)
 //   emission                Algorithm 4  G~[j] <- V[j] (.) Mask
 //   momentum factor masking Sec. 3.3 (V <- V (.) !Mask ; U <- U (.) !Mask)
@@ -111,17 +112,27 @@ void dgc_oracle_clip_coef(int32_t num_tensors, const int64_t* offset, const int6
 
 // Eq. 5 / Algorithm 4: u <- m*u + gc ; v <- v + u, with gc = g*coef.
 // Three (four with clipping) separately rounded fp32 operations per element.
+// nesterov != 0: Algorithm 5 (Appendix B, Eq. 8 with U = m*u): U <- m*(U + gc) ;
+// V <- (V + U) + gc, the sum taken left to right as the algorithm prints it.
 void dgc_oracle_momentum_correction(int32_t num_tensors, const int64_t* offset,
                                     const int64_t* numel, float* u, float* v, const float* g,
-                                    float momentum, float coef) {
+                                    float momentum, float coef, int32_t nesterov) {
   for (int32_t j = 0; j < num_tensors; ++j) {
     const int64_t o = offset[j];
     for (int64_t i = 0; i < numel[j]; ++i) {
       const float gc = g[o + i] * coef;
-      const float t = momentum * u[o + i];
-      const float un = t + gc;
-      u[o + i] = un;
-      v[o + i] = v[o + i] + un;
+      if (nesterov) {
+        const float t = u[o + i] + gc;
+        const float un = momentum * t;
+        u[o + i] = un;
+        const float w = v[o + i] + un;
+        v[o + i] = w + gc;
+      } else {
+        const float t = momentum * u[o + i];
+        const float un = t + gc;
+        u[o + i] = un;
+        v[o + i] = v[o + i] + un;
+      }
     }
   }
 }
@@ -151,6 +162,7 @@ void dgc_oracle_select_topk(int64_t n, const float* v, int64_t k, int64_t* sel_i
 //   k[j]                : number of entries to send from tensor j
 //   out_offset[j]       : where tensor j's pairs start in out_idx/out_val
 //   out_idx             : index into g/u/v (offset[j] + local index), ascending per tensor
+//   nesterov            : non-zero selects Algorithm 5's update instead of Algorithm 4's
 //   coef_override_flag  : when non-zero, coef_override replaces the computed clip
 //                         coefficient (so that state can be compared after two
 //                         implementations rounded the norm differently)
@@ -159,8 +171,8 @@ void dgc_oracle_compress(int32_t num_tensors, const int64_t* offset, const int64
                          const int64_t* k, const int64_t* out_offset, float* u, float* v,
                          const float* g, float momentum, double clip_threshold,
                          int32_t num_workers, int32_t coef_override_flag, float coef_override,
-                         int32_t brute_force, int32_t* out_idx, float* out_val, double* norm_out,
-                         float* coef_out) {
+                         int32_t brute_force, int32_t nesterov, int32_t* out_idx, float* out_val,
+                         double* norm_out, float* coef_out) {
   // Local gradient clipping, before the accumulation.
   double norm = 0.0;
   float coef = 1.0f;
@@ -170,7 +182,7 @@ void dgc_oracle_compress(int32_t num_tensors, const int64_t* offset, const int64
   *coef_out = coef;
 
   // Momentum correction.
-  dgc_oracle_momentum_correction(num_tensors, offset, numel, u, v, g, momentum, coef);
+  dgc_oracle_momentum_correction(num_tensors, offset, numel, u, v, g, momentum, coef, nesterov);
 
   // Per tensor: select, emit, mask.
   std::vector<int64_t> sel;

@@ -49,15 +49,16 @@ def lib() -> ctypes.CDLL:
                                            ctypes.c_int32, _f64p, _f32p]
         L.dgc_oracle_momentum_correction.restype = None
         L.dgc_oracle_momentum_correction.argtypes = [ctypes.c_int32, _i64p, _i64p, _f32p, _f32p,
-                                                     _f32p, ctypes.c_float, ctypes.c_float]
+                                                     _f32p, ctypes.c_float, ctypes.c_float,
+                                                     ctypes.c_int32]
         L.dgc_oracle_select_topk.restype = None
         L.dgc_oracle_select_topk.argtypes = [ctypes.c_int64, _f32p, ctypes.c_int64, _i64p,
                                              ctypes.c_int32]
         L.dgc_oracle_compress.restype = None
         L.dgc_oracle_compress.argtypes = [ctypes.c_int32, _i64p, _i64p, _i64p, _i64p, _f32p, _f32p,
                                           _f32p, ctypes.c_float, ctypes.c_double, ctypes.c_int32,
-                                          ctypes.c_int32, ctypes.c_float, ctypes.c_int32, _i32p,
-                                          _f32p, _f64p, _f32p]
+                                          ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
+                                          ctypes.c_int32, _i32p, _f32p, _f64p, _f32p]
         L.dgc_oracle_decode_accumulate.restype = None
         L.dgc_oracle_decode_accumulate.argtypes = [ctypes.c_int32, ctypes.POINTER(_i32p),
                                                    ctypes.POINTER(_f32p), _i64p, _f32p,
@@ -96,14 +97,16 @@ def clip_coef(offset, numel, g, clip_threshold: float, num_workers: int):
     return norm.value, np.float32(coef.value)
 
 
-def momentum_correction(offset, numel, u, v, g, momentum: float, coef: float) -> None:
+def momentum_correction(offset, numel, u, v, g, momentum: float, coef: float,
+                        nesterov: bool = False) -> None:
     offset = np.ascontiguousarray(offset, dtype=np.int64)
     numel = np.ascontiguousarray(numel, dtype=np.int64)
     lib().dgc_oracle_momentum_correction(len(numel), _p(offset, _i64p), _p(numel, _i64p),
                                          _p(_chk(u, np.float32), _f32p),
                                          _p(_chk(v, np.float32), _f32p),
                                          _p(_chk(g, np.float32), _f32p),
-                                         ctypes.c_float(momentum), ctypes.c_float(coef))
+                                         ctypes.c_float(momentum), ctypes.c_float(coef),
+                                         int(nesterov))
 
 
 def select_topk(v: np.ndarray, k: int, brute_force: bool = False) -> np.ndarray:
@@ -125,13 +128,14 @@ class Worker:
     """State of one worker (u, v) plus the segment table of its gradient set."""
 
     def __init__(self, offset, numel, arena_len: int, num_workers: int, momentum: float,
-                 clip_threshold: float, sparsity: float):
+                 clip_threshold: float, sparsity: float, nesterov: bool = False):
         self.offset = np.ascontiguousarray(offset, dtype=np.int64)
         self.numel = np.ascontiguousarray(numel, dtype=np.int64)
         self.arena_len = int(arena_len)
         self.num_workers = int(num_workers)
         self.momentum = float(momentum)
         self.clip_threshold = float(clip_threshold)
+        self.nesterov = bool(nesterov)
         self.u = np.zeros(self.arena_len, dtype=np.float32)   # Algorithm 4: U <- 0
         self.v = np.zeros(self.arena_len, dtype=np.float32)   # Algorithm 4: V <- 0
         self.set_sparsity(sparsity)
@@ -159,7 +163,8 @@ class Worker:
             ctypes.c_float(self.momentum), self.clip_threshold, self.num_workers,
             int(coef_override is not None),
             ctypes.c_float(0.0 if coef_override is None else float(coef_override)),
-            int(brute_force), _p(idx, _i32p), _p(val, _f32p), ctypes.byref(norm),
+            int(brute_force), int(self.nesterov), _p(idx, _i32p), _p(val, _f32p),
+            ctypes.byref(norm),
             ctypes.byref(coef))
         return CompressResult(idx, val, norm.value, np.float32(coef.value))
 

@@ -35,7 +35,8 @@ class Config(ctypes.Structure):
                 ("tensor_numel", ctypes.POINTER(ctypes.c_int64)), ("momentum", ctypes.c_float),
                 ("clip_threshold", ctypes.c_float), ("sparsity", ctypes.c_double),
                 ("sample_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
-                ("device", ctypes.c_int32), ("debug_sample_rank", ctypes.c_int32)]
+                ("device", ctypes.c_int32), ("debug_sample_rank", ctypes.c_int32),
+                ("nesterov", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class Status(ctypes.Structure):
@@ -63,6 +64,9 @@ _sigs = {
                                                       ctypes.POINTER(_vp), _i64p, _vp,
                                                       ctypes.c_int64, _vp]),
     "dgc_apply_sgd": (ctypes.c_int32, [_vp, _vp, ctypes.c_int64, ctypes.c_float, _vp]),
+    "dgc_decode_apply_sgd": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
+                                              ctypes.POINTER(_vp), _i64p, _vp, ctypes.c_int64,
+                                              ctypes.c_float, _vp, ctypes.c_int64, _vp]),
     "dgc_get_status": (ctypes.c_int32, [_vp, _vp, ctypes.POINTER(Status)]),
     "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
@@ -121,11 +125,12 @@ class State:
 
     def __init__(self, tensor_numel: Sequence[int], num_workers: int, momentum: float,
                  clip_threshold: float, sparsity: float, sample_ratio: float = 0.01,
-                 seed: int = 0, device: int = 0, debug_sample_rank: int = 0):
+                 seed: int = 0, device: int = 0, debug_sample_rank: int = 0,
+                 nesterov: bool = False):
         numel = (ctypes.c_int64 * len(tensor_numel))(*[int(n) for n in tensor_numel])
         cfg = Config(len(tensor_numel), int(num_workers), numel, float(momentum),
                      float(clip_threshold), float(sparsity), float(sample_ratio), int(seed),
-                     int(device), int(debug_sample_rank))
+                     int(device), int(debug_sample_rank), int(bool(nesterov)), 0)
         self._h = _vp()
         self.num_tensors = len(tensor_numel)
         self.device = int(device)
@@ -235,6 +240,21 @@ def decode_accumulate(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[tor
                                       dense_out.numel(), workspace.data_ptr(),
                                       workspace.numel() * workspace.element_size(),
                                       _stream(stream)), "dgc_decode_accumulate")
+
+
+def decode_apply_sgd(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[torch.Tensor],
+                     w: torch.Tensor, lr: float, workspace: torch.Tensor, stream=None,
+                     nnz: Optional[Sequence[int]] = None) -> None:
+    """w <- w - lr * (sum of the workers' sparse lists), touching only the listed entries."""
+    n = len(idx_lists)
+    ip = (_vp * n)(*[_dev(t, torch.int32) for t in idx_lists])
+    vp = (_vp * n)(*[_dev(t, torch.float32) for t in val_lists])
+    cnt = (ctypes.c_int64 * n)(*[int(c) for c in (nnz if nnz is not None
+                                                  else [t.numel() for t in idx_lists])])
+    _check(_lib.dgc_decode_apply_sgd(n, ip, vp, cnt, _dev(w, torch.float32), w.numel(), float(lr),
+                                     workspace.data_ptr(),
+                                     workspace.numel() * workspace.element_size(),
+                                     _stream(stream)), "dgc_decode_apply_sgd")
 
 
 STATIC_DECODE_WORDS = 1 << 18

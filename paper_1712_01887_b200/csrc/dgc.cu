@@ -84,7 +84,7 @@ struct dgc_state {
   // optional timing of the streaming kernel (dgc_profile_enable)
   std::vector<cudaEvent_t> prof_ev;   // 6 events per recorded call (stage boundaries)
   int prof_cap = 0, prof_n = 0;
-  int norm_grid = 0, main_grid = 0, main_grid_clip = 0;
+  int norm_grid = 0;
   int select_smem_keys = 0;
   bool alive = false;
 };
@@ -392,13 +392,6 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   const float one = 1.0f;
   if (cudaMemcpy(st->plan.coef, &one, 4, cudaMemcpyHostToDevice) != cudaSuccess) return fail(DGC_ECUDA);
   // launch geometry
-  int occ = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_update_emit<false>, kMainThreads, 0) !=
-      cudaSuccess) return fail(DGC_ECUDA);
-  st->main_grid = st->sm_count * std::max(occ, 1);
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, k_update_emit<true>, kMainThreads, 0) !=
-      cudaSuccess) return fail(DGC_ECUDA);
-  st->main_grid_clip = st->sm_count * std::max(occ, 1);
   st->norm_grid = std::min(kMaxNormGrid, st->sm_count * 8);
   if (cudaFuncSetAttribute(k_emit_mask, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            kEmitSmemBytes) != cudaSuccess) return fail(DGC_ECUDA);
@@ -457,6 +450,7 @@ int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, f
   cudaStream_t s = as_stream(stream);
   const Plan& p = st->plan;
   const bool clip = st->cfg.clip_threshold > 0.0f;
+  const bool nest = st->cfg.nesterov != 0;
   const float m = st->cfg.momentum;
   const int parity = (int)(st->iterations & 1);
   const uint64_t call_seed = st->cfg.seed * 0x9E3779B97F4A7C15ull + (uint64_t)st->iterations;
@@ -473,15 +467,19 @@ int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, f
   if (prof) DGC_CUDA(cudaEventRecord(ev[1], s));
   if (!st->sample_blocks.empty()) {
     const int grid = (int)st->sample_blocks.size();
-    if (clip) k_sample_threshold<true><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
-    else k_sample_threshold<false><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
+    if (clip && nest) k_sample_threshold<true, true><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
+    else if (clip) k_sample_threshold<true, false><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
+    else if (nest) k_sample_threshold<false, true><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
+    else k_sample_threshold<false, false><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (prof) DGC_CUDA(cudaEventRecord(ev[2], s));
   {
     const int need = (p.num_segs + (kMainThreads / 32) - 1) / (kMainThreads / 32);
-    if (clip) k_update_emit<true><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
-    else k_update_emit<false><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
+    if (clip && nest) k_update_emit<true, true><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
+    else if (clip) k_update_emit<true, false><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
+    else if (nest) k_update_emit<false, true><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
+    else k_update_emit<false, false><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (prof) DGC_CUDA(cudaEventRecord(ev[3], s));
@@ -579,8 +577,39 @@ int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lis
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
   k_decode_bounds<<<dim3(gx, num_workers), 256, 0, s>>>(a, (int32_t*)workspace);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_decode_tiles<<<a.num_tiles, kDecodeThreads, 0, s>>>(a, (const int32_t*)workspace, dense_out,
-                                                       dense_len);
+  k_decode_tiles<false><<<a.num_tiles, kDecodeThreads, 0, s>>>(a, (const int32_t*)workspace,
+                                                              dense_out, dense_len, 0.0f);
+  return check_launch();
+}
+
+int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_lists,
+                             const float* const* val_lists, const int64_t* nnz, float* w,
+                             int64_t len, float lr, void* workspace, int64_t workspace_bytes,
+                             void* stream) {
+  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
+  if (!idx_lists || !val_lists || !nnz || len < 0 || len >= (int64_t)1 << 31) return DGC_EINVAL;
+  if (len == 0) return DGC_OK;
+  if (!w || !workspace) return DGC_EINVAL;
+  if (workspace_bytes < dgc_decode_workspace_bytes(num_workers, len)) return DGC_ECAPACITY;
+  DecodeArgs a{};
+  int64_t max_nnz = 0;
+  for (int k = 0; k < num_workers; ++k) {
+    if (nnz[k] < 0 || nnz[k] > len) return DGC_EINVAL;
+    if (nnz[k] > 0 && (!idx_lists[k] || !val_lists[k])) return DGC_EINVAL;
+    a.idx[k] = idx_lists[k];
+    a.val[k] = val_lists[k];
+    a.nnz[k] = (int32_t)nnz[k];
+    max_nnz = std::max(max_nnz, nnz[k]);
+  }
+  a.num_workers = num_workers;
+  a.num_tiles = (int32_t)((len + kDecodeTile - 1) / kDecodeTile);
+  cudaStream_t s = as_stream(stream);
+  int32_t rc;
+  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
+  k_decode_bounds<<<dim3(gx, num_workers), 256, 0, s>>>(a, (int32_t*)workspace);
+  if ((rc = check_launch()) != DGC_OK) return rc;
+  k_decode_tiles<true><<<a.num_tiles, kDecodeThreads, 0, s>>>(a, (const int32_t*)workspace, w, len,
+                                                             lr);
   return check_launch();
 }
 
@@ -734,6 +763,6 @@ extern "C" int32_t dgc_decode_accumulate_static(int32_t num_workers,
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
   k_decode_bounds<<<dim3(gx, num_workers), 256, 0, s>>>(a, bounds);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_decode_tiles<<<a.num_tiles, kDecodeThreads, 0, s>>>(a, bounds, dense_out, dense_len);
+  k_decode_tiles<false><<<a.num_tiles, kDecodeThreads, 0, s>>>(a, bounds, dense_out, dense_len, 0.0f);
   return check_launch();
 }

@@ -133,13 +133,19 @@ __device__ __forceinline__ T load_record(const T* ptr) {
 // ------------------------------------------------------------------ device helpers
 __device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
 
-// Eq. 5, one element: gc = g*coef ; u <- m*u + gc ; v <- v + u (each rounded once).
-template <bool CLIP>
+// One element of the accumulation, every operation rounded once.
+// Eq. 5 / Algorithm 4:           gc = g*coef ; u <- m*u + gc ; v <- v + u
+// Algorithm 5 (NEST, Appendix B): gc = g*coef ; u <- m*(u + gc) ; v <- (v + u) + gc
+template <bool CLIP, bool NEST>
 __device__ __forceinline__ void mc_step(float g, float coef, float m, float& u, float& v) {
   const float gc = CLIP ? __fmul_rn(g, coef) : g;
-  const float t = __fmul_rn(m, u);
-  u = __fadd_rn(t, gc);
-  v = __fadd_rn(v, u);
+  if (NEST) {
+    u = __fmul_rn(m, __fadd_rn(u, gc));
+    v = __fadd_rn(__fadd_rn(v, u), gc);
+  } else {
+    u = __fadd_rn(__fmul_rn(m, u), gc);
+    v = __fadd_rn(v, u);
+  }
 }
 
 __device__ __forceinline__ uint64_t mix64(uint64_t x) {
@@ -342,7 +348,7 @@ k_sumsq(Plan p, const float* __restrict__ g, double thr_local, int clip_on) {
 // selects.  r is small against the sample, so that block first bounds the
 // answer from below by the rank-r of the per-thread maxima (at least r keys
 // reach it), keeps the few keys that reach the bound and selects among them.
-template <bool CLIP>
+template <bool CLIP, bool NEST>
 __global__ void __launch_bounds__(kSampleThreads)
 k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_seed) {
   __shared__ uint32_t hist[kHistWords(kSampleThreads)];
@@ -370,10 +376,10 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
       const float4 gg = __ldg(reinterpret_cast<const float4*>(g) + pos);
       float4 u = __ldcg(reinterpret_cast<const float4*>(p.u) + pos);
       float4 v = __ldcg(reinterpret_cast<const float4*>(p.v) + pos);
-      mc_step<CLIP>(gg.x, coef, m, u.x, v.x);
-      mc_step<CLIP>(gg.y, coef, m, u.y, v.y);
-      mc_step<CLIP>(gg.z, coef, m, u.z, v.z);
-      mc_step<CLIP>(gg.w, coef, m, u.w, v.w);
+      mc_step<CLIP, NEST>(gg.x, coef, m, u.x, v.x);
+      mc_step<CLIP, NEST>(gg.y, coef, m, u.y, v.y);
+      mc_step<CLIP, NEST>(gg.z, coef, m, u.z, v.z);
+      mc_step<CLIP, NEST>(gg.w, coef, m, u.w, v.w);
       gkeys[s] = make_uint4(mag_key(v.x), mag_key(v.y), mag_key(v.z), mag_key(v.w));
     }
   }
@@ -477,7 +483,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
 // bytes per warp load), keeps everything in registers, and appends the
 // segment's candidates -- in ascending index order -- to its part's list with
 // one integer atomicAdd per segment that has any.
-template <bool CLIP>
+template <bool CLIP, bool NEST>
 __global__ void __launch_bounds__(kMainThreads)
 k_update_emit(Plan p, const float* __restrict__ g, float m) {
   const int lane = threadIdx.x & 31;
@@ -506,10 +512,10 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
     uint32_t flags = 0;   // bit (4*i + c): element c of float4 i is a candidate
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      mc_step<CLIP>(gg[i].x, coef, m, uu[i].x, vv[i].x);
-      mc_step<CLIP>(gg[i].y, coef, m, uu[i].y, vv[i].y);
-      mc_step<CLIP>(gg[i].z, coef, m, uu[i].z, vv[i].z);
-      mc_step<CLIP>(gg[i].w, coef, m, uu[i].w, vv[i].w);
+      mc_step<CLIP, NEST>(gg[i].x, coef, m, uu[i].x, vv[i].x);
+      mc_step<CLIP, NEST>(gg[i].y, coef, m, uu[i].y, vv[i].y);
+      mc_step<CLIP, NEST>(gg[i].z, coef, m, uu[i].z, vv[i].z);
+      mc_step<CLIP, NEST>(gg[i].w, coef, m, uu[i].w, vv[i].w);
       flags |= (uint32_t)(mag_key(vv[i].x) >= thr) << (4 * i + 0);
       flags |= (uint32_t)(mag_key(vv[i].y) >= thr) << (4 * i + 1);
       flags |= (uint32_t)(mag_key(vv[i].z) >= thr) << (4 * i + 2);
@@ -1267,41 +1273,102 @@ k_decode_bounds(const __grid_constant__ DecodeArgs a, int32_t* __restrict__ boun
   }
 }
 
+// SGD = false: the tile of the dense gradient is written out (zero-fill fused).
+// SGD = true (Eq. 5, third term applied directly): `dense` is the weight array; only the
+// entries some worker lists are updated, w <- w - lr * G with G summed as above -- bit for bit
+// what the dense gradient followed by k_sgd gives, because w - lr * (+0) = w.
+template <bool SGD>
 __global__ void __launch_bounds__(kDecodeThreads)
 k_decode_tiles(const __grid_constant__ DecodeArgs a, const int32_t* __restrict__ bounds,
-               float* __restrict__ dense, long long dense_len) {
+               float* __restrict__ dense, long long dense_len, float lr) {
   __shared__ float tile[kDecodeTile];
-  __shared__ int s_lo[DGC_MAX_DECODE_WORKERS], s_hi[DGC_MAX_DECODE_WORKERS];
+  __shared__ uint32_t touched[kDecodeTile / 32];
+  __shared__ int s_lo[DGC_MAX_DECODE_WORKERS];
+  __shared__ int s_cum[DGC_MAX_DECODE_WORKERS + 1];   // pairs of workers 0..w-1 inside this tile
   const int t = blockIdx.x;
+  const int tid = threadIdx.x;
   const long long base = (long long)t * kDecodeTile;
-  if (threadIdx.x < a.num_workers) {
-    const int32_t* b = bounds + (size_t)threadIdx.x * (a.num_tiles + 1);
-    s_lo[threadIdx.x] = __ldg(b + t);
-    s_hi[threadIdx.x] = __ldg(b + t + 1);
+  const int N = a.num_workers;
+  if (tid < 32) {
+    // the tile's slice of every worker list, and the running pair count in worker order
+    int run = 0;
+    for (int w0 = 0; w0 < N; w0 += 32) {
+      const int w = w0 + tid;
+      int lo = 0, len = 0;
+      if (w < N) {
+        const int32_t* b = bounds + (size_t)w * (a.num_tiles + 1);
+        lo = __ldg(b + t);
+        len = __ldg(b + t + 1) - lo;
+        s_lo[w] = lo;
+      }
+      const int incl = warp_incl_scan(len);
+      if (w < N) s_cum[w] = run + incl - len;
+      run += __shfl_sync(0xFFFFFFFFu, incl, 31);
+    }
+    if (tid == 0) s_cum[N] = run;
+  }
+  if (SGD) {
+    __syncthreads();
+    if (s_cum[N] == 0) return;                    // nothing listed in this tile: w is unchanged
+    if (tid < kDecodeTile / 32) touched[tid] = 0u;
   }
 #pragma unroll
-  for (int i = threadIdx.x; i < kDecodeTile; i += kDecodeThreads) tile[i] = 0.0f;
+  for (int i = tid; i < kDecodeTile; i += kDecodeThreads) tile[i] = 0.0f;
   __syncthreads();
-  for (int w = 0; w < a.num_workers; ++w) {
-    const int lo = s_lo[w], hi = s_hi[w];
-    if (hi > lo) {      // block-uniform
-      const int32_t* idx = a.idx[w];
-      const float* val = a.val[w];
-      for (int i = lo + threadIdx.x; i < hi; i += kDecodeThreads) {
-        const int l = __ldg(idx + i) - (int)base;
-        tile[l] = __fadd_rn(tile[l], __ldg(val + i));
+  const int total = s_cum[N];
+  // pairs in (worker, position) order, a block's worth at a time: all loads of a chunk are
+  // issued together, then the adds run one worker after the other (worker order, and no two
+  // threads touch one slot between barriers because indices are unique within a worker)
+  for (int q0 = 0; q0 < total; q0 += kDecodeThreads) {
+    const int q = q0 + tid;
+    int myw = -1, l = 0;
+    float v = 0.0f;
+    if (q < total) {
+      int lo = 0, hi = N;                        // largest w with s_cum[w] <= q
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (s_cum[mid] <= q) lo = mid; else hi = mid;
       }
+      myw = lo;
+      const int pos = s_lo[lo] + (q - s_cum[lo]);
+      l = __ldg(a.idx[lo] + pos) - (int)base;
+      v = __ldg(a.val[lo] + pos);
+    }
+    // workers present in this chunk (block-uniform bounds)
+    int wfirst = 0, wlast = N - 1;
+    {
+      const int qa = q0, qb = min(q0 + kDecodeThreads, total) - 1;
+      int lo = 0, hi = N;
+      while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_cum[mid] <= qa) lo = mid; else hi = mid; }
+      wfirst = lo;
+      lo = 0; hi = N;
+      while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_cum[mid] <= qb) lo = mid; else hi = mid; }
+      wlast = lo;
+    }
+    for (int w = wfirst; w <= wlast; ++w) {
+      if (myw == w) tile[l] = __fadd_rn(tile[l], v);
       __syncthreads();
     }
+    if (SGD && myw >= 0) atomicOr(&touched[l >> 5], 1u << (l & 31));
+  }
+  if (SGD) {
+    __syncthreads();
+    for (int i = tid; i < kDecodeTile; i += kDecodeThreads) {
+      if ((touched[i >> 5] >> (i & 31)) & 1u) {
+        float* wp = dense + base + i;
+        *wp = __fsub_rn(*wp, __fmul_rn(lr, tile[i]));
+      }
+    }
+    return;
   }
   const long long rem = dense_len - base;
   if (rem >= kDecodeTile) {
     float4* d4 = reinterpret_cast<float4*>(dense + base);
     const float4* t4 = reinterpret_cast<const float4*>(tile);
 #pragma unroll
-    for (int i = threadIdx.x; i < kDecodeTile / 4; i += kDecodeThreads) __stcs(d4 + i, t4[i]);
+    for (int i = tid; i < kDecodeTile / 4; i += kDecodeThreads) __stcs(d4 + i, t4[i]);
   } else {
-    for (int i = threadIdx.x; i < (int)rem; i += kDecodeThreads) dense[base + i] = tile[i];
+    for (int i = tid; i < (int)rem; i += kDecodeThreads) dense[base + i] = tile[i];
   }
 }
 

@@ -38,11 +38,11 @@ class Pair:
 
     def __init__(self, numel: Sequence[int], num_workers: int, momentum: float, clip: float,
                  sparsity: float, seed: int = 0, sample_ratio: float = 0.01,
-                 debug_sample_rank: int = 0):
+                 debug_sample_rank: int = 0, nesterov: bool = False):
         self.gpu = B.State(numel, num_workers, momentum, clip, sparsity, sample_ratio=sample_ratio,
-                           seed=seed, debug_sample_rank=debug_sample_rank)
+                           seed=seed, debug_sample_rank=debug_sample_rank, nesterov=nesterov)
         self.cpu = O.Worker(self.gpu.arena_offset, numel, self.gpu.arena_len, num_workers,
-                            momentum, clip, sparsity)
+                            momentum, clip, sparsity, nesterov=nesterov)
         self.clip = clip
         self.numel = list(numel)
         self._alloc_out()
@@ -135,4 +135,8 @@ def receive_side(idx_lists, val_lists, dense_len: int, w_init: np.ndarray, lr: f
     wref = w_init.copy()
     O.apply_sgd(wref, ref, lr)
     _assert_bits(wd.cpu().numpy(), wref, "weights after SGD")
+    # the fused form (Eq. 5 third term applied to the listed entries only) must give the same bits
+    wf = torch.from_numpy(w_init.copy()).cuda()
+    B.decode_apply_sgd(di, dv, wf, lr, ws)
+    _assert_bits(wf.cpu().numpy(), wref, "weights after fused sparse decode + SGD")
     return ref, wref

@@ -19,10 +19,11 @@ def P():
 
 
 def _run_workload(P, wl, iterations, workers=None, seed=0, receive=True, schedule=None,
-                  check_state=True):
+                  check_state=True, nesterov=False):
     N = workers or wl.num_workers
     pairs = [P.Pair(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold, wl.sparsity,
-                    seed=seed + w, sample_ratio=wl.sample_ratio) for w in range(N)]
+                    seed=seed + w, sample_ratio=wl.sample_ratio, nesterov=nesterov)
+             for w in range(N)]
     rep = P.ParityReport()
     off, L = pairs[0].gpu.arena_offset, pairs[0].gpu.arena_len
     rng = np.random.default_rng(99)
@@ -76,6 +77,18 @@ def test_deepspeech_small_warmup_schedule(P):
     wl = I.workload("deepspeech_small")
     stages = [0.75, 0.9375, 0.984375, 0.996, 0.999]
     _run_workload(P, wl, 10, workers=2, schedule=lambda t: stages[min(t // 2, 4)])
+
+
+def test_nesterov_variant_deepspeech_small(P):
+    """Algorithm 5 (the paper trains its speech model with Nesterov momentum and clipping)."""
+    wl = I.workload("deepspeech_small")
+    wl.sparsity = 0.999
+    _run_workload(P, wl, 4, workers=2, nesterov=True)
+
+
+def test_nesterov_variant_resnet50_no_clip(P):
+    wl = I.workload("resnet50")
+    _run_workload(P, wl, 2, workers=1, receive=False, nesterov=True)
 
 
 def test_lstm_full_size_one_worker(P):

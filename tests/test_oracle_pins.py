@@ -39,6 +39,46 @@ def test_alg4_two_iterations_trace(golden_dir):
             assert r.coef == np.float32(1.0)
 
 
+def test_alg5_nesterov_trace(golden_dir):
+    G = _load(golden_dir, "alg5_nesterov_two_iterations.json")
+    w = O.Worker([0], [G["n"]], G["n"], 1, G["momentum"], 0.0, G["sparsity"], nesterov=True)
+    assert w.k.tolist() == [G["k"]]
+    for it in G["iterations"]:
+        r = w.compress(_f32(it["g"]))
+        assert r.idx.tolist() == it["sent_idx"]
+        assert r.val.tolist() == it["sent_val"]
+        assert w.u.tolist() == it["u_after"]
+        assert w.v.tolist() == it["v_after"]
+
+
+def test_nesterov_matches_eq8_parametrisation():
+    """Appendix B, Eq. 8: u' = m u + g ; v' = v + (m u' + g).  Algorithm 5 stores U = m u'.
+    A float64 shadow of Eq. 8 must track the oracle's Algorithm 5 state on unsent entries."""
+    rng = np.random.default_rng(13)
+    n, T, m = 50, 10, 0.9
+    w = O.Worker([0], [n], n, 1, m, 0.0, 0.98, nesterov=True)      # k = 1
+    G = rng.standard_normal((T, n)).astype(np.float32)
+    G[:, 7] = 1e6
+    u_eq = np.zeros(n)
+    v_eq = np.zeros(n)
+    for t in range(T):
+        r = w.compress(G[t].copy())
+        assert r.idx.tolist() == [7]
+        u_eq = m * u_eq + G[t].astype(np.float64)
+        v_eq = v_eq + (m * u_eq + G[t].astype(np.float64))
+    keep = np.arange(n) != 7
+    np.testing.assert_allclose(w.u[keep], (m * u_eq)[keep], rtol=2e-5, atol=1e-6)
+    np.testing.assert_allclose(w.v[keep], v_eq[keep], rtol=2e-5, atol=1e-6)
+    # constant gradient closed form: u_eq,t = g (1 - m^t)/(1 - m); v_T = sum_t (m u_eq,t + g)
+    w2 = O.Worker([0], [4], 4, 1, 0.5, 0.0, 0.75, nesterov=True)
+    g = _f32([0.25, 0.25, 0.25, 4096.0])
+    for t in range(1, 7):
+        w2.compress(g.copy())
+        u_t = [0.25 * (1 - 0.5 ** i) / 0.5 for i in range(1, t + 1)]
+        assert w2.u[0] == np.float32(0.5 * u_t[-1])
+        assert w2.v[0] == np.float32(sum(0.5 * x + 0.25 for x in u_t))
+
+
 def test_tie_goes_to_lower_index(golden_dir):
     G = _load(golden_dir, "tie_rule.json")
     for brute in (False, True):
