@@ -274,6 +274,13 @@ def run_ours(args):
                "fused_sparse_decode_sgd_ms": _time(
                    lambda: B.decode_apply_sgd(out_i, out_v, weights, LR, ws))}
 
+    # the paper's wire format (values + 16-bit zero run lengths) of one worker's list
+    runs, _vals = B.encode_runlength(out_i[0], out_v[0], L)
+    enc_ms = _time(lambda: B.encode_runlength(out_i[0], out_v[0], L), reps=5)
+    wire = {"entries": int(runs.numel()), "bytes": int(runs.numel()) * 6,
+            "compression_ratio": total * 4 / max(int(runs.numel()) * 6, 1),
+            "encode_ms_with_count_readback": enc_ms}
+
     # end to end through the host-buffer entry point: H2D of every gradient and D2H of the
     # sparse lists inside the timed region
     e2e = None
@@ -342,7 +349,7 @@ def run_ours(args):
         "compress": {"ms_per_worker": compress_ms, "elements_per_s": total / (compress_ms * 1e-3),
                      "algorithmic_gbs": compress_bytes / (compress_ms * 1e-3) / 1e9,
                      "frac_of_peak": compress_bytes / (compress_ms * 1e-3) / 1e9 / peak},
-        "receive": receive, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
+        "receive": receive, "wire_format": wire, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
     }
     print(json.dumps(line))
     if world > 1:

@@ -202,6 +202,34 @@ int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_list
                              int64_t len, float lr, void* workspace, int64_t workspace_bytes,
                              void* stream);
 
+/* Sec. 3.1, encode(): "packs the 32-bit nonzero gradient values and 16-bit run lengths of
+ * zeros" -- the wire format behind the compression ratios of Tables 3 and 4.  Entry t is
+ * (runs_out[t], values_out[t]): skip runs_out[t] zeros, then store values_out[t].  More
+ * than 65535 zeros in a row are bridged by filler entries (65535, +0.0f), each standing for
+ * 65535 zeros and one explicit zero (the paper gives no rule for that case).  Zeros after
+ * the last entry are not encoded.  Encoded size = 6 bytes per entry.
+ *   idx, val      device, nnz pairs, idx strictly ascending (what dgc_compress emits)
+ *   runs_out      device, capacity uint16;  values_out  device, capacity floats
+ *   capacity      >= dgc_runlength_max_entries(nnz, dense_len) always suffices; entries
+ *                 beyond capacity are dropped (never written) and still counted
+ *   count_out     device int64: entries the encoding has (fillers included)
+ *   workspace     device, >= dgc_runlength_workspace_bytes(nnz) bytes, 8-byte aligned
+ * Asynchronous on `stream`. */
+int32_t dgc_encode_runlength(const int32_t* idx, const float* val, int64_t nnz,
+                             uint16_t* runs_out, float* values_out, int64_t capacity,
+                             int64_t* count_out, void* workspace, int64_t workspace_bytes,
+                             void* stream);
+
+/* The inverse: entry t lands at index sum_{j<t} (runs[j] + 1) + runs[t].  Writes `count`
+ * (index, value) pairs, ascending (fillers come back as explicit zeros, which a sum
+ * ignores), ready for dgc_decode_accumulate, and the position after the last entry to
+ * *dense_len_out (device int64).  workspace >= dgc_runlength_workspace_bytes(count). */
+int32_t dgc_decode_runlength(const uint16_t* runs, const float* values, int64_t count,
+                             int32_t* idx_out, float* val_out, int64_t* dense_len_out,
+                             void* workspace, int64_t workspace_bytes, void* stream);
+int64_t dgc_runlength_max_entries(int64_t nnz, int64_t dense_len);
+int64_t dgc_runlength_workspace_bytes(int64_t entries);
+
 /* Synchronises `stream`, then reports counters of the last dgc_compress. */
 int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out);
 

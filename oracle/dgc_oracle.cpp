@@ -223,4 +223,49 @@ void dgc_oracle_apply_sgd(float* w, const float* dense_grad, int64_t len, float 
   }
 }
 
+// Sec. 3.1: "The encode() function packs the 32-bit nonzero gradient values and 16-bit
+// run lengths of zeros."  Entry t = (run_t, value_t): run_t zeros are skipped, then value_t
+// is stored.  The paper gives no rule for more than 65535 zeros in a row; the reading used
+// here bridges the gap with filler entries (65535, +0.0f), each standing for 65535 zeros
+// followed by one slot that holds an explicit zero.  Zeros after the last entry are not
+// encoded (the receiver knows the dense length).
+// idx ascending, no duplicates.  Returns the number of entries written, or -1 if
+// `capacity` is too small.  Encoded size = 6 bytes per entry.
+int64_t dgc_oracle_encode_runlength(const int32_t* idx, const float* val, int64_t nnz,
+                                    uint16_t* runs, float* values, int64_t capacity) {
+  int64_t out = 0;
+  int64_t pos = 0;                       // next dense position not yet accounted for
+  for (int64_t i = 0; i < nnz; ++i) {
+    int64_t gap = static_cast<int64_t>(idx[i]) - pos;     // zeros before this entry
+    while (gap > 65535) {
+      if (out >= capacity) return -1;
+      runs[out] = 65535;
+      values[out] = 0.0f;
+      ++out;
+      gap -= 65536;                      // 65535 zeros and the filler's own slot
+    }
+    if (out >= capacity) return -1;
+    runs[out] = static_cast<uint16_t>(gap);
+    values[out] = val[i];
+    ++out;
+    pos = static_cast<int64_t>(idx[i]) + 1;
+  }
+  return out;
+}
+
+// The inverse: entry t lands at position sum_{j<t} (run_j + 1) + run_t.  Fillers come back
+// as explicit (index, +0.0f) pairs (they cannot be told from a sent zero), which a sum
+// ignores.  Returns the number of pairs (= count).
+int64_t dgc_oracle_decode_runlength(const uint16_t* runs, const float* values, int64_t count,
+                                    int32_t* idx, float* val) {
+  int64_t pos = 0;
+  for (int64_t t = 0; t < count; ++t) {
+    pos += runs[t];
+    idx[t] = static_cast<int32_t>(pos);
+    val[t] = values[t];
+    pos += 1;
+  }
+  return count;
+}
+
 }  // extern "C"

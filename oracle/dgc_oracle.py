@@ -65,6 +65,13 @@ def lib() -> ctypes.CDLL:
                                                    ctypes.c_int64]
         L.dgc_oracle_apply_sgd.restype = None
         L.dgc_oracle_apply_sgd.argtypes = [_f32p, _f32p, ctypes.c_int64, ctypes.c_float]
+        L.dgc_oracle_encode_runlength.restype = ctypes.c_int64
+        L.dgc_oracle_encode_runlength.argtypes = [_i32p, _f32p, ctypes.c_int64,
+                                                  ctypes.POINTER(ctypes.c_uint16), _f32p,
+                                                  ctypes.c_int64]
+        L.dgc_oracle_decode_runlength.restype = ctypes.c_int64
+        L.dgc_oracle_decode_runlength.argtypes = [ctypes.POINTER(ctypes.c_uint16), _f32p,
+                                                  ctypes.c_int64, _i32p, _f32p]
         _lib = L
     return _lib
 
@@ -186,3 +193,27 @@ def apply_sgd(w: np.ndarray, dense_grad: np.ndarray, lr: float) -> None:
     dense_grad = _chk(dense_grad, np.float32)
     assert w.size == dense_grad.size
     lib().dgc_oracle_apply_sgd(_p(w, _f32p), _p(dense_grad, _f32p), w.size, ctypes.c_float(lr))
+
+
+def encode_runlength(idx: np.ndarray, val: np.ndarray, capacity: int):
+    """Sec. 3.1 encode(): (uint16 zero run lengths, float32 values); raises if capacity is short."""
+    idx = _chk(np.ascontiguousarray(idx), np.int32)
+    val = _chk(np.ascontiguousarray(val), np.float32)
+    runs = np.empty(capacity, dtype=np.uint16)
+    values = np.empty(capacity, dtype=np.float32)
+    n = lib().dgc_oracle_encode_runlength(_p(idx, _i32p), _p(val, _f32p), idx.size,
+                                          runs.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16)),
+                                          _p(values, _f32p), int(capacity))
+    if n < 0:
+        raise ValueError("capacity too small")
+    return runs[:n].copy(), values[:n].copy()
+
+
+def decode_runlength(runs: np.ndarray, values: np.ndarray):
+    runs = _chk(np.ascontiguousarray(runs), np.uint16)
+    values = _chk(np.ascontiguousarray(values), np.float32)
+    idx = np.empty(runs.size, dtype=np.int32)
+    val = np.empty(runs.size, dtype=np.float32)
+    lib().dgc_oracle_decode_runlength(runs.ctypes.data_as(ctypes.POINTER(ctypes.c_uint16)),
+                                      _p(values, _f32p), runs.size, _p(idx, _i32p), _p(val, _f32p))
+    return idx, val

@@ -67,6 +67,12 @@ _sigs = {
     "dgc_decode_apply_sgd": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
                                               ctypes.POINTER(_vp), _i64p, _vp, ctypes.c_int64,
                                               ctypes.c_float, _vp, ctypes.c_int64, _vp]),
+    "dgc_encode_runlength": (ctypes.c_int32, [_vp, _vp, ctypes.c_int64, _vp, _vp, ctypes.c_int64,
+                                              _vp, _vp, ctypes.c_int64, _vp]),
+    "dgc_decode_runlength": (ctypes.c_int32, [_vp, _vp, ctypes.c_int64, _vp, _vp, _vp, _vp,
+                                              ctypes.c_int64, _vp]),
+    "dgc_runlength_max_entries": (ctypes.c_int64, [ctypes.c_int64, ctypes.c_int64]),
+    "dgc_runlength_workspace_bytes": (ctypes.c_int64, [ctypes.c_int64]),
     "dgc_get_status": (ctypes.c_int32, [_vp, _vp, ctypes.POINTER(Status)]),
     "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
@@ -255,6 +261,46 @@ def decode_apply_sgd(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[torc
                                      workspace.data_ptr(),
                                      workspace.numel() * workspace.element_size(),
                                      _stream(stream)), "dgc_decode_apply_sgd")
+
+
+def runlength_max_entries(nnz: int, dense_len: int) -> int:
+    return int(_lib.dgc_runlength_max_entries(int(nnz), int(dense_len)))
+
+
+def encode_runlength(idx: torch.Tensor, val: torch.Tensor, dense_len: int, stream=None):
+    """Sec. 3.1 encode(): returns (runs uint16, values float32) device tensors trimmed to the
+    encoded length (synchronises to read the count)."""
+    nnz = idx.numel()
+    cap = runlength_max_entries(nnz, dense_len)
+    runs = torch.empty(cap, dtype=torch.uint16, device=idx.device)
+    values = torch.empty(cap, dtype=torch.float32, device=idx.device)
+    count = torch.zeros(1, dtype=torch.int64, device=idx.device)
+    ws = torch.empty(max(int(_lib.dgc_runlength_workspace_bytes(nnz)), 8), dtype=torch.uint8,
+                     device=idx.device)
+    _check(_lib.dgc_encode_runlength(_dev(idx, torch.int32) if nnz else None,
+                                     _dev(val, torch.float32) if nnz else None, nnz,
+                                     runs.data_ptr(), values.data_ptr(), cap, count.data_ptr(),
+                                     ws.data_ptr(), ws.numel(), _stream(stream)),
+           "dgc_encode_runlength")
+    n = int(count.item())
+    return runs[:n], values[:n]
+
+
+def decode_runlength(runs: torch.Tensor, values: torch.Tensor, stream=None):
+    """Inverse of encode_runlength: (idx int32, val float32, dense position after the last entry)."""
+    n = runs.numel()
+    idx = torch.empty(n, dtype=torch.int32, device=runs.device)
+    val = torch.empty(n, dtype=torch.float32, device=runs.device)
+    end = torch.zeros(1, dtype=torch.int64, device=runs.device)
+    ws = torch.empty(max(int(_lib.dgc_runlength_workspace_bytes(n)), 8), dtype=torch.uint8,
+                     device=runs.device)
+    if not (runs.is_cuda and runs.dtype == torch.uint16 and runs.is_contiguous()):
+        raise ValueError("expected a contiguous CUDA uint16 tensor")
+    _check(_lib.dgc_decode_runlength(runs.data_ptr() if n else None,
+                                     _dev(values, torch.float32) if n else None, n,
+                                     idx.data_ptr(), val.data_ptr(), end.data_ptr(), ws.data_ptr(),
+                                     ws.numel(), _stream(stream)), "dgc_decode_runlength")
+    return idx, val, int(end.item())
 
 
 STATIC_DECODE_WORDS = 1 << 18

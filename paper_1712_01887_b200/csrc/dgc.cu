@@ -613,6 +613,64 @@ int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_list
   return check_launch();
 }
 
+int64_t dgc_runlength_max_entries(int64_t nnz, int64_t dense_len) {
+  if (nnz < 0 || dense_len < 0) return DGC_EINVAL;
+  return nnz + dense_len / 65536 + 1;
+}
+
+int64_t dgc_runlength_workspace_bytes(int64_t entries) {
+  if (entries < 0) return DGC_EINVAL;
+  return ((entries + kRleBlock - 1) / kRleBlock + 1) * 8;
+}
+
+int32_t dgc_encode_runlength(const int32_t* idx, const float* val, int64_t nnz,
+                             uint16_t* runs_out, float* values_out, int64_t capacity,
+                             int64_t* count_out, void* workspace, int64_t workspace_bytes,
+                             void* stream) {
+  if (nnz < 0 || capacity < 0 || !count_out) return DGC_EINVAL;
+  cudaStream_t s = as_stream(stream);
+  int32_t rc;
+  if (nnz == 0) {
+    DGC_CUDA(cudaMemsetAsync(count_out, 0, 8, s));
+    return DGC_OK;
+  }
+  if (!idx || !val || !runs_out || !values_out || !workspace) return DGC_EINVAL;
+  if (workspace_bytes < dgc_runlength_workspace_bytes(nnz)) return DGC_ECAPACITY;
+  if (capacity < nnz) return DGC_ECAPACITY;
+  const int nblocks = (int)((nnz + kRleBlock - 1) / kRleBlock);
+  unsigned long long* sums = (unsigned long long*)workspace;
+  k_rle_block_sums<true><<<nblocks, kRleThreads, 0, s>>>(idx, nullptr, nnz, sums);
+  if ((rc = check_launch()) != DGC_OK) return rc;
+  k_rle_scan_sums<<<1, 1024, 0, s>>>(sums, nblocks, nnz, (long long*)count_out);
+  if ((rc = check_launch()) != DGC_OK) return rc;
+  k_rle_write<true><<<nblocks, kRleThreads, 0, s>>>(idx, val, nullptr, nnz, sums, runs_out,
+                                                    values_out, nullptr, capacity);
+  return check_launch();
+}
+
+int32_t dgc_decode_runlength(const uint16_t* runs, const float* values, int64_t count,
+                             int32_t* idx_out, float* val_out, int64_t* dense_len_out,
+                             void* workspace, int64_t workspace_bytes, void* stream) {
+  if (count < 0) return DGC_EINVAL;
+  cudaStream_t s = as_stream(stream);
+  int32_t rc;
+  if (count == 0) {
+    if (dense_len_out) DGC_CUDA(cudaMemsetAsync(dense_len_out, 0, 8, s));
+    return DGC_OK;
+  }
+  if (!runs || !values || !idx_out || !val_out || !workspace || !dense_len_out) return DGC_EINVAL;
+  if (workspace_bytes < dgc_runlength_workspace_bytes(count)) return DGC_ECAPACITY;
+  const int nblocks = (int)((count + kRleBlock - 1) / kRleBlock);
+  unsigned long long* sums = (unsigned long long*)workspace;
+  k_rle_block_sums<false><<<nblocks, kRleThreads, 0, s>>>(nullptr, runs, count, sums);
+  if ((rc = check_launch()) != DGC_OK) return rc;
+  k_rle_scan_sums<<<1, 1024, 0, s>>>(sums, nblocks, 0, (long long*)dense_len_out);
+  if ((rc = check_launch()) != DGC_OK) return rc;
+  k_rle_write<false><<<nblocks, kRleThreads, 0, s>>>(nullptr, values, runs, count, sums, nullptr,
+                                                     val_out, idx_out, count);
+  return check_launch();
+}
+
 int32_t dgc_apply_sgd(float* w, const float* dense_grad, int64_t len, float lr, void* stream) {
   if (len < 0) return DGC_EINVAL;
   if (len == 0) return DGC_OK;

@@ -1394,4 +1394,140 @@ k_sgd(float* __restrict__ w, const float* __restrict__ G, long long len, float l
   }
 }
 
+// ------------------------------------------------------------------ wire format: values + 16-bit zero run lengths
+// Sec. 3.1: encode() packs the 32-bit non-zero values and 16-bit run lengths of zeros.
+// Entry t = (run_t, value_t): run_t zeros are skipped, then value_t is stored.  A gap of
+// more than 65535 zeros is bridged by filler entries (65535, +0.0f), each standing for 65535
+// zeros and one slot holding an explicit zero (the paper gives no rule; this is the reading).
+// Both directions are an exclusive prefix sum over the list -- fillers per entry when
+// encoding, run + 1 when decoding -- done as block sums, one block scanning the block sums,
+// and a write pass (three launches, no block waits for another).
+constexpr int kRleThreads = 256;
+constexpr int kRlePer = 4;                         // entries per thread
+constexpr int kRleBlock = kRleThreads * kRlePer;   // entries per block
+
+// ENCODE: x_i = fillers before entry i = (zeros before it) >> 16.   DECODE: x_t = run_t + 1.
+template <bool ENCODE>
+__device__ __forceinline__ uint32_t rle_term(const int32_t* idx, const uint16_t* runs, long long i) {
+  if (ENCODE) {
+    const long long prev = i == 0 ? -1 : (long long)__ldg(idx + i - 1);
+    return (uint32_t)(((long long)__ldg(idx + i) - prev - 1) >> 16);
+  }
+  return (uint32_t)__ldg(runs + i) + 1u;
+}
+
+template <bool ENCODE>
+__global__ void __launch_bounds__(kRleThreads)
+k_rle_block_sums(const int32_t* __restrict__ idx, const uint16_t* __restrict__ runs, long long n,
+                 unsigned long long* __restrict__ block_sums) {
+  __shared__ unsigned long long swarp[kRleThreads / 32];
+  const long long base = (long long)blockIdx.x * kRleBlock + threadIdx.x * kRlePer;
+  unsigned long long s = 0;
+#pragma unroll
+  for (int q = 0; q < kRlePer; ++q)
+    if (base + q < n) s += rle_term<ENCODE>(idx, runs, base + q);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  if ((threadIdx.x & 31) == 0) swarp[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    unsigned long long t = 0;
+    for (int w = 0; w < kRleThreads / 32; ++w) t += swarp[w];
+    block_sums[blockIdx.x] = t;
+  }
+}
+
+// One block: exclusive scan of the block sums in place; total (plus `add`) to *total_out.
+__global__ void __launch_bounds__(1024)
+k_rle_scan_sums(unsigned long long* __restrict__ block_sums, int nblocks, long long add,
+                long long* __restrict__ total_out) {
+  __shared__ unsigned long long swarp[32];
+  __shared__ unsigned long long s_run;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_run = 0;
+  __syncthreads();
+  for (int b0 = 0; b0 < nblocks; b0 += 1024) {
+    const int b = b0 + tid;
+    const unsigned long long x = b < nblocks ? block_sums[b] : 0ull;
+    unsigned long long incl = x;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += t;
+    }
+    if (lane == 31) swarp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const unsigned long long w = swarp[lane];
+      unsigned long long wi = w;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, wi, o);
+        if (lane >= o) wi += t;
+      }
+      swarp[lane] = wi - w;
+    }
+    __syncthreads();
+    const unsigned long long run = s_run;
+    const unsigned long long ex = run + swarp[warp] + incl - x;
+    if (b < nblocks) block_sums[b] = ex;
+    __syncthreads();
+    if (tid == 1023) s_run = ex + x;
+    __syncthreads();
+  }
+  if (tid == 0) *total_out = (long long)s_run + add;
+}
+
+template <bool ENCODE>
+__global__ void __launch_bounds__(kRleThreads)
+k_rle_write(const int32_t* __restrict__ idx, const float* __restrict__ val,
+            const uint16_t* __restrict__ runs, long long n,
+            const unsigned long long* __restrict__ block_sums, uint16_t* __restrict__ runs_out,
+            float* __restrict__ values_out, int32_t* __restrict__ idx_out, long long capacity) {
+  __shared__ unsigned long long swarp[kRleThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long base = (long long)blockIdx.x * kRleBlock + tid * kRlePer;
+  uint32_t x[kRlePer];
+  unsigned long long s = 0;
+#pragma unroll
+  for (int q = 0; q < kRlePer; ++q) {
+    x[q] = base + q < n ? rle_term<ENCODE>(idx, runs, base + q) : 0u;
+    s += x[q];
+  }
+  unsigned long long incl = s;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  if (lane == 31) swarp[warp] = incl;
+  __syncthreads();
+  unsigned long long before = block_sums[blockIdx.x] + incl - s;
+  for (int w = 0; w < warp; ++w) before += swarp[w];
+#pragma unroll
+  for (int q = 0; q < kRlePer; ++q) {
+    const long long i = base + q;
+    if (i < n) {
+      if (ENCODE) {
+        // entry i goes after the `before` fillers of earlier entries and its own x fillers
+        long long o = i + (long long)before;
+        for (uint32_t f = 0; f < x[q]; ++f, ++o) {
+          if (o < capacity) { runs_out[o] = 65535; values_out[o] = 0.0f; }
+        }
+        const long long prev = i == 0 ? -1 : (long long)__ldg(idx + i - 1);
+        const long long gap = (long long)__ldg(idx + i) - prev - 1;
+        if (o < capacity) {
+          runs_out[o] = (uint16_t)(gap - ((long long)x[q] << 16));
+          values_out[o] = __ldg(val + i);
+        }
+      } else {
+        // entry i sits run_i positions after everything before it
+        idx_out[i] = (int32_t)((long long)before + (long long)x[q] - 1);
+        values_out[i] = __ldg(val + i);
+      }
+    }
+    before += x[q];
+  }
+}
+
 }  // namespace dgc

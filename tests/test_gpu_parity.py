@@ -323,3 +323,62 @@ def test_decode_edge_cases(P):
             val.append(rng.standard_normal(i.size).astype(np.float32))
         w0 = rng.standard_normal(L).astype(np.float32)
         P.receive_side(idx, val, L, w0, lr=0.05)
+
+
+def test_runlength_wire_format_matches_oracle(P):
+    """Sec. 3.1 encode(): values + 16-bit zero run lengths, against the oracle bit for bit;
+    then back through decode and the dense sum."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    rng = np.random.default_rng(31)
+    cases = [(1000, 0), (1000, 1000), (70000, 2), (5_000_000, 5000), (300_000_000, 9),
+             (40_000_000, 3_000_000)]
+    for L, k in cases:
+        if k == 0:
+            idx = np.zeros(0, np.int32)
+        elif k < 100:
+            idx = np.sort(rng.choice(L, size=k, replace=False)).astype(np.int32)
+        else:
+            idx = np.sort(rng.choice(L, size=k, replace=False)).astype(np.int32)
+        val = rng.standard_normal(idx.size).astype(np.float32)
+        cap = B.runlength_max_entries(idx.size, L)
+        ref_runs, ref_vals = O.encode_runlength(idx, val, cap)
+        di, dv = torch.from_numpy(idx).cuda(), torch.from_numpy(val).cuda()
+        runs, values = B.encode_runlength(di, dv, L)
+        assert runs.cpu().numpy().tobytes() == ref_runs.tobytes(), (L, k)
+        assert values.cpu().numpy().tobytes() == ref_vals.tobytes(), (L, k)
+        ridx, rval = O.decode_runlength(ref_runs, ref_vals)
+        gi, gv, end = B.decode_runlength(runs, values)
+        assert gi.cpu().numpy().tobytes() == ridx.tobytes()
+        assert gv.cpu().numpy().tobytes() == rval.tobytes()
+        assert end == (int(idx[-1]) + 1 if idx.size else 0)
+
+
+def test_runlength_of_compressed_resnet50_gradient(P):
+    """The lists dgc_compress emits, encoded: size against the paper's Table 3 context
+    (ResNet-50: 97.49 MB -> 0.35 MB, 277x) and decoded back into the same dense sum."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    wl = I.workload("resnet50")
+    st = B.State(wl.numel, 8, 0.9, 0.0, 0.999, seed=1)
+    L, off = st.arena_len, st.arena_offset
+    g = np.zeros(L, np.float32)
+    I.fill(wl, g, off, 0, 0)
+    oi = torch.empty(st.max_nnz, dtype=torch.int32, device="cuda")
+    ov = torch.empty(st.max_nnz, dtype=torch.float32, device="cuda")
+    st.compress(torch.from_numpy(g).cuda(), oi, ov)
+    runs, values = B.encode_runlength(oi, ov, L)
+    ref_runs, ref_vals = O.encode_runlength(oi.cpu().numpy(), ov.cpu().numpy(),
+                                            B.runlength_max_entries(st.max_nnz, L))
+    assert runs.cpu().numpy().tobytes() == ref_runs.tobytes()
+    assert values.cpu().numpy().tobytes() == ref_vals.tobytes()
+    ratio = wl.total * 4 / (runs.numel() * 6)
+    assert 600 < ratio < 667          # 25,670 entries of 6 bytes for 102 MB: about 664x
+    gi, gv, _ = B.decode_runlength(runs, values)
+    dense_a = torch.empty(L, dtype=torch.float32, device="cuda")
+    dense_b = torch.empty(L, dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.decode_workspace_bytes(1, L), dtype=torch.uint8, device="cuda")
+    B.decode_accumulate([oi], [ov], dense_a, ws)
+    B.decode_accumulate([gi], [gv], dense_b, ws)
+    assert torch.equal(dense_a.view(torch.int32), dense_b.view(torch.int32))
+    st.close()

@@ -422,3 +422,39 @@ def test_end_to_end_matches_dense_momentum_sgd_when_everything_is_eventually_sen
         u[r.idx] = 0
         sent[r.idx] += r.val
         assert np.array_equal(sent + w.v, acc)
+
+
+# ------------------------------------------------------------------ encode(): values + 16-bit zero runs
+
+def test_encode_runlength_hand_example(golden_dir):
+    G = _load(golden_dir, "encode_runlength.json")
+    runs, values = O.encode_runlength(np.asarray(G["idx"], np.int32), _f32(G["val"]), 16)
+    assert runs.tolist() == G["runs"] and values.tolist() == G["values"]
+    idx, val = O.decode_runlength(runs, values)
+    assert idx.tolist() == G["decoded_idx"] and val.tolist() == G["values"]
+    with pytest.raises(ValueError):
+        O.encode_runlength(np.asarray(G["idx"], np.int32), _f32(G["val"]), 5)
+
+
+def test_encode_runlength_round_trip_and_size():
+    rng = np.random.default_rng(77)
+    for L, k in ((1000, 0), (1000, 1000), (5_000_000, 5000), (3_000_000, 7), (70000, 2)):
+        idx = np.sort(rng.choice(L, size=k, replace=False)).astype(np.int32)
+        val = rng.standard_normal(k).astype(np.float32)
+        runs, values = O.encode_runlength(idx, val, k + L // 65536 + 1)
+        # fillers: one per full 65536 positions of every gap
+        gaps = np.diff(np.concatenate([[-1], idx.astype(np.int64)])) - 1
+        assert runs.size == k + int((gaps // 65536).sum())
+        di, dv = O.decode_runlength(runs, values)
+        dense = np.zeros(L, np.float32)
+        dense[idx] = val
+        back = np.zeros(L, np.float32)
+        back[di] = dv
+        assert back.tobytes() == dense.tobytes()
+        assert np.all(np.diff(di) > 0)
+    # compression ratio of a 99.9 %-sparse vector stays below the format's bound 4/(6*0.001)
+    L, k = 2_000_000, 2000
+    idx = np.sort(rng.choice(L, size=k, replace=False)).astype(np.int32)
+    runs, values = O.encode_runlength(idx, np.ones(k, np.float32), k + 64)
+    ratio = 4 * L / (6 * runs.size)
+    assert 600 < ratio <= 4 / (6 * 0.001) + 1e-9
