@@ -393,7 +393,7 @@ def cpu_baseline(wl, budget_s=20.0):
         step(n + 1)
         n += 1
         dt = time.perf_counter() - t0
-        if dt >= budget_s or n >= 8:
+        if dt >= budget_s or n >= 64:
             break
     return {"value": nw * wl.total * n / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
             "sample": f"{n} step(s) of {nw} simulated worker(s) on the full {wl.name} shapes "
@@ -440,7 +440,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50",

@@ -382,3 +382,61 @@ def test_runlength_of_compressed_resnet50_gradient(P):
     B.decode_accumulate([gi], [gv], dense_b, ws)
     assert torch.equal(dense_a.view(torch.int32), dense_b.view(torch.int32))
     st.close()
+
+
+def test_workers_on_four_streams_like_the_benchmark(P):
+    """bench.py issues the simulated workers' compress calls round robin on four CUDA streams
+    and joins them before the decode.  Same launch configuration here, on the ResNet-50-shaped
+    set with all 8 workers: every worker must still match its oracle bit for bit."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    wl = I.workload("resnet50")
+    NW, NS, T = 8, 4, 2
+    states = [B.State(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold, wl.sparsity,
+                      seed=I.BASE_SEED + w) for w in range(NW)]
+    L, off = states[0].arena_len, states[0].arena_offset
+    oracles = [O.Worker(off, wl.numel, L, wl.num_workers, wl.momentum, wl.clip_threshold,
+                        wl.sparsity) for _ in range(NW)]
+    nnz = states[0].max_nnz
+    main = torch.cuda.current_stream()
+    side = [torch.cuda.Stream() for _ in range(NS)]
+    out_i = [torch.empty(nnz, dtype=torch.int32, device="cuda") for _ in range(NW)]
+    out_v = [torch.empty(nnz, dtype=torch.float32, device="cuda") for _ in range(NW)]
+    dense = torch.empty(L, dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.decode_workspace_bytes(NW, L), dtype=torch.uint8, device="cuda")
+    weights = torch.zeros(L, dtype=torch.float32, device="cuda")
+    w_ref = np.zeros(L, np.float32)
+    for t in range(T):
+        hosts = []
+        for w in range(NW):
+            g = np.zeros(L, np.float32)
+            I.fill(wl, g, off, worker=w, iteration=t)
+            hosts.append(g)
+        dev = [torch.from_numpy(g).cuda() for g in hosts]
+        torch.cuda.synchronize()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        for s_ in side:
+            s_.wait_event(fork)
+        for w in range(NW):
+            states[w].compress(dev[w], out_i[w], out_v[w], stream=side[w % NS])
+        for s_ in side:
+            e = torch.cuda.Event()
+            e.record(s_)
+            main.wait_event(e)
+        B.decode_accumulate(out_i, out_v, dense, ws)
+        B.apply_sgd(weights, dense, 0.1)
+        torch.cuda.synchronize()
+        res = [oracles[w].compress(hosts[w]) for w in range(NW)]
+        for w in range(NW):
+            assert out_i[w].cpu().numpy().tobytes() == res[w].idx.tobytes(), (t, w)
+            assert out_v[w].cpu().numpy().tobytes() == res[w].val.tobytes(), (t, w)
+        ref = O.decode_accumulate([r.idx for r in res], [r.val for r in res], L)
+        O.apply_sgd(w_ref, ref, 0.1)
+        assert dense.cpu().numpy().tobytes() == ref.tobytes()
+        assert weights.cpu().numpy().tobytes() == w_ref.tobytes()
+    for w in (0, NW - 1):
+        u, v = states[w].read()
+        assert u.tobytes() == oracles[w].u.tobytes() and v.tobytes() == oracles[w].v.tobytes()
+    for st in states:
+        st.close()
