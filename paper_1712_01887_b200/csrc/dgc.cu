@@ -308,6 +308,23 @@ int32_t upload_plan(dgc_state* st, bool first) {
 
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
+// Launch with the programmatic-dependent-launch attribute (see pdl_enter in the kernels).
+template <class... KArgs, class... Args>
+inline void launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                   Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // error: check_launch()
+}
+
 int32_t check_launch() {
   g_launches.fetch_add(1, std::memory_order_relaxed);
   cudaError_t e = cudaGetLastError();
@@ -461,44 +478,44 @@ int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, f
   if (clip) {
     const double thr_local =
         (double)st->cfg.clip_threshold / std::sqrt((double)st->cfg.num_workers);
-    k_sumsq<<<st->norm_grid, kNormThreads, 0, s>>>(p, grad_arena, thr_local, 1);
+    launch(k_sumsq, st->norm_grid, kNormThreads, 0, s, p, grad_arena, thr_local, 1);
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (prof) DGC_CUDA(cudaEventRecord(ev[1], s));
   if (!st->sample_blocks.empty()) {
     const int grid = (int)st->sample_blocks.size();
-    if (clip && nest) k_sample_threshold<true, true><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
-    else if (clip) k_sample_threshold<true, false><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
-    else if (nest) k_sample_threshold<false, true><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
-    else k_sample_threshold<false, false><<<grid, kSampleThreads, 0, s>>>(p, grad_arena, m, call_seed);
+    if (clip && nest) launch(k_sample_threshold<true, true>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
+    else if (clip) launch(k_sample_threshold<true, false>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
+    else if (nest) launch(k_sample_threshold<false, true>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
+    else launch(k_sample_threshold<false, false>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (prof) DGC_CUDA(cudaEventRecord(ev[2], s));
   {
     const int need = (p.num_segs + (kMainThreads / 32) - 1) / (kMainThreads / 32);
-    if (clip && nest) k_update_emit<true, true><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
-    else if (clip) k_update_emit<true, false><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
-    else if (nest) k_update_emit<false, true><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
-    else k_update_emit<false, false><<<need, kMainThreads, 0, s>>>(p, grad_arena, m);
+    if (clip && nest) launch(k_update_emit<true, true>, need, kMainThreads, 0, s, p, grad_arena, m);
+    else if (clip) launch(k_update_emit<true, false>, need, kMainThreads, 0, s, p, grad_arena, m);
+    else if (nest) launch(k_update_emit<false, true>, need, kMainThreads, 0, s, p, grad_arena, m);
+    else launch(k_update_emit<false, false>, need, kMainThreads, 0, s, p, grad_arena, m);
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (prof) DGC_CUDA(cudaEventRecord(ev[3], s));
-  k_select<<<p.num_tensors, kSelectThreads,
-             (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s>>>(
-      p, st->select_smem_keys, parity);
+  launch(k_select, p.num_tensors, kSelectThreads,
+         (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s, p, st->select_smem_keys,
+         parity);
   if ((rc = check_launch()) != DGC_OK) return rc;
   if (p.num_big_parts > 0) {
-    k_big_hist<0><<<p.num_big_parts, kBigThreads, 0, s>>>(p);
+    launch(k_big_hist<0>, p.num_big_parts, kBigThreads, 0, s, p);
     if ((rc = check_launch()) != DGC_OK) return rc;
-    k_big_hist<1><<<p.num_big_parts, kBigThreads, 0, s>>>(p);
+    launch(k_big_hist<1>, p.num_big_parts, kBigThreads, 0, s, p);
     if ((rc = check_launch()) != DGC_OK) return rc;
-    k_big_hist<2><<<p.num_big_parts, kBigThreads, 0, s>>>(p);
+    launch(k_big_hist<2>, p.num_big_parts, kBigThreads, 0, s, p);
     if ((rc = check_launch()) != DGC_OK) return rc;
-    k_big_final<<<p.num_big_tensors, kSelectThreads, 0, s>>>(p, parity);
+    launch(k_big_final, p.num_big_tensors, kSelectThreads, 0, s, p, parity);
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (prof) DGC_CUDA(cudaEventRecord(ev[4], s));
-  k_emit_mask<<<p.num_parts, kEmitThreads, kEmitSmemBytes, s>>>(p, out_idx, out_val);
+  launch(k_emit_mask, p.num_parts, kEmitThreads, kEmitSmemBytes, s, p, out_idx, out_val);
   if ((rc = check_launch()) != DGC_OK) return rc;
   if (prof) {
     DGC_CUDA(cudaEventRecord(ev[5], s));
@@ -575,9 +592,9 @@ int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lis
   cudaStream_t s = as_stream(stream);
   int32_t rc;
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
-  k_decode_bounds<<<dim3(gx, num_workers), 256, 0, s>>>(a, (int32_t*)workspace);
+  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_decode_tiles<false><<<a.num_tiles, kDecodeThreads, 0, s>>>(a, (const int32_t*)workspace,
+  launch(k_decode_tiles<false>, a.num_tiles, kDecodeThreads, 0, s, a, (const int32_t*)workspace,
                                                               dense_out, dense_len, 0.0f);
   return check_launch();
 }
@@ -606,9 +623,9 @@ int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_list
   cudaStream_t s = as_stream(stream);
   int32_t rc;
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
-  k_decode_bounds<<<dim3(gx, num_workers), 256, 0, s>>>(a, (int32_t*)workspace);
+  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_decode_tiles<true><<<a.num_tiles, kDecodeThreads, 0, s>>>(a, (const int32_t*)workspace, w, len,
+  launch(k_decode_tiles<true>, a.num_tiles, kDecodeThreads, 0, s, a, (const int32_t*)workspace, w, len,
                                                              lr);
   return check_launch();
 }
@@ -639,11 +656,11 @@ int32_t dgc_encode_runlength(const int32_t* idx, const float* val, int64_t nnz,
   if (capacity < nnz) return DGC_ECAPACITY;
   const int nblocks = (int)((nnz + kRleBlock - 1) / kRleBlock);
   unsigned long long* sums = (unsigned long long*)workspace;
-  k_rle_block_sums<true><<<nblocks, kRleThreads, 0, s>>>(idx, nullptr, nnz, sums);
+  launch(k_rle_block_sums<true>, nblocks, kRleThreads, 0, s, idx, nullptr, nnz, sums);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_rle_scan_sums<<<1, 1024, 0, s>>>(sums, nblocks, nnz, (long long*)count_out);
+  launch(k_rle_scan_sums, 1, 1024, 0, s, sums, nblocks, nnz, (long long*)count_out);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_rle_write<true><<<nblocks, kRleThreads, 0, s>>>(idx, val, nullptr, nnz, sums, runs_out,
+  launch(k_rle_write<true>, nblocks, kRleThreads, 0, s, idx, val, nullptr, nnz, sums, runs_out,
                                                     values_out, nullptr, capacity);
   return check_launch();
 }
@@ -662,11 +679,11 @@ int32_t dgc_decode_runlength(const uint16_t* runs, const float* values, int64_t 
   if (workspace_bytes < dgc_runlength_workspace_bytes(count)) return DGC_ECAPACITY;
   const int nblocks = (int)((count + kRleBlock - 1) / kRleBlock);
   unsigned long long* sums = (unsigned long long*)workspace;
-  k_rle_block_sums<false><<<nblocks, kRleThreads, 0, s>>>(nullptr, runs, count, sums);
+  launch(k_rle_block_sums<false>, nblocks, kRleThreads, 0, s, nullptr, runs, count, sums);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_rle_scan_sums<<<1, 1024, 0, s>>>(sums, nblocks, 0, (long long*)dense_len_out);
+  launch(k_rle_scan_sums, 1, 1024, 0, s, sums, nblocks, 0, (long long*)dense_len_out);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_rle_write<false><<<nblocks, kRleThreads, 0, s>>>(nullptr, values, runs, count, sums, nullptr,
+  launch(k_rle_write<false>, nblocks, kRleThreads, 0, s, nullptr, values, runs, count, sums, nullptr,
                                                      val_out, idx_out, count);
   return check_launch();
 }
@@ -679,7 +696,7 @@ int32_t dgc_apply_sgd(float* w, const float* dense_grad, int64_t len, float lr, 
     return DGC_EINVAL;
   const int64_t n4 = std::max<int64_t>(len >> 2, 1);
   const int grid = (int)std::min<int64_t>((n4 + 255) / 256, 148 * 16);
-  k_sgd<<<grid, 256, 0, as_stream(stream)>>>(w, dense_grad, len, lr);
+  launch(k_sgd, grid, 256, 0, as_stream(stream), w, dense_grad, len, lr);
   return check_launch();
 }
 
@@ -819,8 +836,8 @@ extern "C" int32_t dgc_decode_accumulate_static(int32_t num_workers,
   cudaStream_t s = as_stream(stream);
   int32_t rc;
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
-  k_decode_bounds<<<dim3(gx, num_workers), 256, 0, s>>>(a, bounds);
+  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, bounds);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  k_decode_tiles<false><<<a.num_tiles, kDecodeThreads, 0, s>>>(a, bounds, dense_out, dense_len, 0.0f);
+  launch(k_decode_tiles<false>, a.num_tiles, kDecodeThreads, 0, s, a, bounds, dense_out, dense_len, 0.0f);
   return check_launch();
 }
