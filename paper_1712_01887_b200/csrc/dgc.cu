@@ -76,6 +76,7 @@ struct dgc_state {
   int32_t* d_cand_idx = nullptr;
   float* d_cand_val = nullptr;
   int64_t cand_alloc = 0;
+  uint32_t* d_sent_bits = nullptr;
   float* d_stage_g = nullptr;     // dgc_compress_host staging
   int32_t* d_stage_idx = nullptr;
   float* d_stage_val = nullptr;
@@ -116,6 +117,12 @@ void dev_free(dgc_state* st, void* ptr) {
 
 // Everything that depends on the sparsity: k, output offsets, sampling plan,
 // candidate capacities.  Segments and parts depend only on the shapes.
+// Scattered zeroing of u and v at the sent entries costs a sector read and write per touched
+// 32-byte sector and array; recording one bit per element and zeroing in the next call's
+// streaming pass costs 0.25 B/element flat.  The bitmap wins when more than about one entry
+// in 512 is sent.
+int defer_mask_for(double sparsity) { return (1.0 - sparsity) > 1.0 / 512.0 ? 1 : 0; }
+
 // Keys one k_select block may hold in shared memory: two blocks per SM when there are more
 // tensors than SMs, else one large block.
 int select_key_cap(const dgc_state* st) {
@@ -331,6 +338,13 @@ int32_t check_launch() {
   return e == cudaSuccess ? DGC_OK : DGC_ECUDA;
 }
 
+int32_t flush_pending_mask(dgc_state* st, cudaStream_t s) {
+  if (!st->plan.defer_mask) return DGC_OK;
+  const long long words = st->arena_len / 32;
+  launch(k_apply_pending_mask, 1184, 256, 0, s, st->plan, words);
+  return check_launch();
+}
+
 }  // namespace
 
 // ====================================================================== C ABI
@@ -394,6 +408,11 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   st->plan.u = (float*)ptr;
   if ((rc = dev_alloc(st, &ptr, (size_t)st->arena_len * 4)) != DGC_OK) return fail(rc);
   st->plan.v = (float*)ptr;
+  if ((rc = dev_alloc(st, &ptr, (size_t)st->arena_len / 8)) != DGC_OK) return fail(rc);
+  st->d_sent_bits = (uint32_t*)ptr;
+  st->plan.sent_bits = st->d_sent_bits;
+  if (cudaMemset(ptr, 0, (size_t)st->arena_len / 8) != cudaSuccess) return fail(DGC_ECUDA);
+  st->plan.defer_mask = defer_mask_for(st->sparsity);
   // scalars: partials[kMaxNormGrid] doubles, norm, diag[8] long long, coef, ticket
   const size_t scal_bytes = (kMaxNormGrid + 1) * 8 + 8 * 8 + 16;
   if ((rc = dev_alloc(st, &ptr, scal_bytes)) != DGC_OK) return fail(rc);
@@ -434,9 +453,14 @@ int32_t dgc_set_sparsity(dgc_state* st, double sparsity) {
   if (!st || !st->alive) return DGC_ESTATE;
   if (!(sparsity >= 0.0 && sparsity < 1.0)) return DGC_EINVAL;
   DGC_CUDA(cudaSetDevice(st->device));
+  int32_t rc = flush_pending_mask(st, nullptr);   // entries sent by the last call, if deferred
+  if (rc != DGC_OK) return rc;
   DGC_CUDA(cudaDeviceSynchronize());
   build_host_plan(st, sparsity);
-  return upload_plan(st, false);
+  rc = upload_plan(st, false);
+  st->plan.sent_bits = st->d_sent_bits;
+  st->plan.defer_mask = defer_mask_for(sparsity);
+  return rc;
 }
 
 int64_t dgc_max_nnz(const dgc_state* st) {
@@ -762,6 +786,8 @@ int32_t dgc_profile_read(dgc_state* st, float* ms_out, int32_t capacity, int32_t
 int32_t dgc_state_read(dgc_state* st, float* u_host, float* v_host, void* stream) {
   if (!st || !st->alive) return DGC_ESTATE;
   cudaStream_t s = as_stream(stream);
+  const int32_t frc = flush_pending_mask(st, s);
+  if (frc != DGC_OK) return frc;
   const size_t bytes = (size_t)st->arena_len * 4;
   if (u_host) DGC_CUDA(cudaMemcpyAsync(u_host, st->plan.u, bytes, cudaMemcpyDeviceToHost, s));
   if (v_host) DGC_CUDA(cudaMemcpyAsync(v_host, st->plan.v, bytes, cudaMemcpyDeviceToHost, s));
@@ -772,6 +798,8 @@ int32_t dgc_state_read(dgc_state* st, float* u_host, float* v_host, void* stream
 int32_t dgc_state_write(dgc_state* st, const float* u_host, const float* v_host, void* stream) {
   if (!st || !st->alive) return DGC_ESTATE;
   cudaStream_t s = as_stream(stream);
+  const int32_t frc = flush_pending_mask(st, s);   // pending zeroing belongs to the old contents
+  if (frc != DGC_OK) return frc;
   const size_t bytes = (size_t)st->arena_len * 4;
   if (u_host) DGC_CUDA(cudaMemcpyAsync(st->plan.u, u_host, bytes, cudaMemcpyHostToDevice, s));
   if (v_host) DGC_CUDA(cudaMemcpyAsync(st->plan.v, v_host, bytes, cudaMemcpyHostToDevice, s));

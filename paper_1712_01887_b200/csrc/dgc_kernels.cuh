@@ -115,6 +115,10 @@ struct Plan {
   long long* diag;           // [2][4]: flags, full_select, candidates, unused
   float* u;
   float* v;
+  // deferred masking (low sparsity): k_emit_mask records the sent entries as one bit each and
+  // the next call's kernels zero u and v at those entries in registers before using them
+  uint32_t* sent_bits;       // arena_len / 32 words, 16 per segment
+  int32_t defer_mask;        // 1: masking is deferred through sent_bits
   int32_t num_tensors, num_parts, num_segs;
   int32_t num_big_parts, num_big_tensors;
 };
@@ -389,6 +393,14 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
       const float4 gg = __ldg(reinterpret_cast<const float4*>(g) + pos);
       float4 u = __ldcg(reinterpret_cast<const float4*>(p.u) + pos);
       float4 v = __ldcg(reinterpret_cast<const float4*>(p.v) + pos);
+      if (p.defer_mask) {
+        // entries sent by the previous call are still to be zeroed
+        const uint32_t nib = (__ldcg(p.sent_bits + (pos >> 3)) >> ((pos & 7u) * 4u)) & 0xFu;
+        if (nib & 1u) { u.x = 0.0f; v.x = 0.0f; }
+        if (nib & 2u) { u.y = 0.0f; v.y = 0.0f; }
+        if (nib & 4u) { u.z = 0.0f; v.z = 0.0f; }
+        if (nib & 8u) { u.w = 0.0f; v.w = 0.0f; }
+      }
       mc_step<CLIP, NEST>(gg.x, coef, m, u.x, v.x);
       mc_step<CLIP, NEST>(gg.y, coef, m, u.y, v.y);
       mc_step<CLIP, NEST>(gg.z, coef, m, u.z, v.z);
@@ -525,6 +537,20 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
     const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
     const int end = pm.end;
     const bool full = base + kSeg <= end;
+    if (p.defer_mask) {
+      // Sec. 3.3 masking of the previous call, applied here: the segment's 512 sent bits are 16
+      // words; element c of float4 (i, lane) is bit (lane & 7) * 4 + c of word 4 * i + lane / 8
+      const uint32_t myword = lane < 16 ? __ldcg(p.sent_bits + seg * 16 + lane) : 0u;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t w = __shfl_sync(0xFFFFFFFFu, myword, i * 4 + (lane >> 3));
+        const uint32_t nib = (w >> ((lane & 7) * 4)) & 0xFu;
+        if (nib & 1u) { uu[i].x = 0.0f; vv[i].x = 0.0f; }
+        if (nib & 2u) { uu[i].y = 0.0f; vv[i].y = 0.0f; }
+        if (nib & 4u) { uu[i].z = 0.0f; vv[i].z = 0.0f; }
+        if (nib & 8u) { uu[i].w = 0.0f; vv[i].w = 0.0f; }
+      }
+    }
     uint32_t flags = 0;   // bit (4*i + c): element c of float4 i is a candidate
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -1149,6 +1175,12 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   if (ps.dense) {
     __syncthreads();
     if (tid == 0) p.p_count[part] = 0;
+    if (p.defer_mask && tid < pm.nseg) {
+      // the full-selection path zeroes u and v itself: nothing is pending for this part
+      uint4* dst = reinterpret_cast<uint4*>(p.sent_bits + (size_t)(pm.seg0 + tid) * 16);
+#pragma unroll
+      for (int w = 0; w < 4; ++w) dst[w] = make_uint4(0u, 0u, 0u, 0u);
+    }
     if (pm.first) {
       const TensorMeta t = load_record(p.tm + pm.tensor);
       dense_select_emit(p, t, pm.tensor, out_idx, out_val, smask, sh);
@@ -1241,8 +1273,10 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
     const int idx = pm.seg0 * kSeg + local;
     out_idx[pos] = idx;
     out_val[pos] = val;
-    p.u[idx] = 0.0f;
-    p.v[idx] = 0.0f;
+    if (!p.defer_mask) {
+      p.u[idx] = 0.0f;
+      p.v[idx] = 0.0f;
+    }
   };
 #pragma unroll
   for (int b = 0; b < kEmitRegs; ++b)
@@ -1261,6 +1295,48 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
       const int i = i0 + b * kEmitThreads + tid;
       const uint32_t key = mag_key(v4[b]);
       if (i < count && key >= kth) emit(x4[b] - pm.seg0 * kSeg, v4[b], key);
+    }
+  }
+  if (p.defer_mask && tid < pm.nseg) {
+    // record what was sent from segment `tid`: all "greater" bits and the tied bits within
+    // the quota (lowest indices first); the next call zeroes u and v there
+    int left = max(0, quota - s_eqb[tid]);
+    uint32_t words[16];
+#pragma unroll
+    for (int w = 0; w < 16; ++w) {
+      uint32_t e = meq[tid * kMaskStride + w];
+      uint32_t taken = 0;
+      while (e != 0 && left > 0) {
+        const uint32_t low = e & (0u - e);
+        taken |= low;
+        e ^= low;
+        --left;
+      }
+      words[w] = mgt[tid * kMaskStride + w] | taken;
+    }
+    uint4* dst = reinterpret_cast<uint4*>(p.sent_bits + (size_t)(pm.seg0 + tid) * 16);
+#pragma unroll
+    for (int w = 0; w < 4; ++w)
+      dst[w] = make_uint4(words[4 * w], words[4 * w + 1], words[4 * w + 2], words[4 * w + 3]);
+  }
+}
+
+// Applies (and clears) whatever k_emit_mask left in sent_bits: u = v = 0 at the recorded
+// entries.  Used when the state is read out or the masking mode changes.
+__global__ void __launch_bounds__(256)
+k_apply_pending_mask(Plan p, long long words) {
+  pdl_enter();
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long w = (long long)blockIdx.x * blockDim.x + threadIdx.x; w < words; w += stride) {
+    uint32_t bits = p.sent_bits[w];
+    if (bits) {
+      p.sent_bits[w] = 0u;
+      while (bits) {
+        const int b = __ffs(bits) - 1;
+        bits &= bits - 1;
+        p.u[w * 32 + b] = 0.0f;
+        p.v[w * 32 + b] = 0.0f;
+      }
     }
   }
 }

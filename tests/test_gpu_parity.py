@@ -440,3 +440,32 @@ def test_workers_on_four_streams_like_the_benchmark(P):
         assert u.tobytes() == oracles[w].u.tobytes() and v.tobytes() == oracles[w].v.tobytes()
     for st in states:
         st.close()
+
+
+@pytest.mark.parametrize("sparsity", [0.75, 0.9375, 0.99])
+def test_deferred_masking_without_reading_state_between_iterations(P, sparsity):
+    """Below 99.8 % sparsity the library does not zero u and v at the sent entries right away:
+    it records them as bits and the next call's kernels zero them in registers.  Reading the
+    state flushes that, so here nothing is read until the end: five iterations compared on
+    indices and values only (with exact ties in the data), then the final state."""
+    numel = [300000, 70001, 513, 1 << 20]
+    pair = P.Pair(numel, 2, 0.9, 1.0, sparsity, seed=11)
+    rep = P.ParityReport()
+    rng = np.random.default_rng(23)
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    for t in range(5):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for j, (o, n) in enumerate(zip(off, numel)):
+            if j == 1:      # quantised: many ties at the threshold
+                g[o:o + n] = rng.integers(-3, 4, size=n).astype(np.float32) * np.float32(0.125)
+            else:
+                g[o:o + n] = rng.standard_normal(n).astype(np.float32)
+        pair.step(g, rep, check_state=False)
+    u, v = pair.gpu.read()
+    assert u.tobytes() == pair.cpu.u.tobytes() and v.tobytes() == pair.cpu.v.tobytes()
+    # and once more after the flush: the next call must start from the flushed state
+    g = P.arena_with_padding_poison(L, off, numel)
+    for o, n in zip(off, numel):
+        g[o:o + n] = rng.standard_normal(n).astype(np.float32)
+    pair.step(g, rep, check_state=True)
+    pair.close()
