@@ -401,6 +401,83 @@ def cpu_baseline(wl, budget_s=20.0):
             "host_cpus": os.cpu_count()}
 
 
+def run_schedule(args):
+    """The warm-up schedule of Sec. 4.1 on one workload (BASELINE config 4: 5 stages of
+    `--stage-iters` iterations at 75 %, 93.75 %, 98.4375 %, 99.6 %, 99.9 % sparsity): the same
+    step as the headline benchmark, timed per stage, dgc_set_sparsity between stages."""
+    import torch
+    from paper_1712_01887_b200 import build
+    build.build()
+    from paper_1712_01887_b200 import binding as B
+    wl = I.workload(args.workload)
+    if args.clip is not None:
+        wl.clip_threshold = args.clip
+    NW = args.workers or wl.num_workers
+    off, L, hosts = _make_pool(wl, NW, 0)
+    states = [B.State(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold,
+                      B.warmup_sparsity(0), sample_ratio=wl.sample_ratio, seed=I.BASE_SEED + w)
+              for w in range(NW)]
+    pool = [[h.cuda() for h in row] for row in hosts]
+    dense = torch.empty(L, dtype=torch.float32, device="cuda")
+    weights = torch.randn(L, dtype=torch.float32, device="cuda")
+    ws = torch.empty(max(B.decode_workspace_bytes(NW, L), 4), dtype=torch.uint8, device="cuda")
+    main_stream = torch.cuda.current_stream()
+    NS = max(1, min(args.streams, NW))
+    side = [torch.cuda.Stream() for _ in range(NS)] if NS > 1 else [main_stream]
+    peak, _ = _peaks()
+    rows = []
+    it = 0
+    for stage in range(5):
+        s_ = B.warmup_sparsity(stage)
+        for st in states:
+            st.set_sparsity(s_)
+        nnz = states[0].max_nnz
+        out_i = [torch.empty(nnz, dtype=torch.int32, device="cuda") for _ in range(NW)]
+        out_v = [torch.empty(nnz, dtype=torch.float32, device="cuda") for _ in range(NW)]
+
+        def step(t):
+            if NS > 1:
+                ev = torch.cuda.Event()
+                ev.record(main_stream)
+                for q in side:
+                    q.wait_event(ev)
+            for w in range(NW):
+                states[w].compress(pool[w][t % POOL], out_i[w], out_v[w], stream=side[w % NS])
+            if NS > 1:
+                for q in side:
+                    ev = torch.cuda.Event()
+                    ev.record(q)
+                    main_stream.wait_event(ev)
+            B.decode_accumulate(out_i, out_v, dense, ws)
+            B.apply_sgd(weights, dense, LR)
+
+        for _ in range(3):
+            step(it)
+            it += 1
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.stage_iters):
+            step(it)
+            it += 1
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / args.stage_iters
+        nbytes = NW * ((24.0 if wl.clip_threshold > 0 else 20.0) * wl.total + 16.0 * nnz) + \
+            4.0 * L + 8.0 * NW * nnz + 12.0 * L
+        rows.append({"stage": stage, "sparsity": s_, "nnz_per_worker": nnz, "ms_per_step": ms,
+                     "elements_per_s": NW * wl.total / (ms * 1e-3),
+                     "algorithmic_gbs": nbytes / (ms * 1e-3) / 1e9,
+                     "frac_of_peak": nbytes / (ms * 1e-3) / 1e9 / peak})
+    total_ms = sum(r["ms_per_step"] for r in rows) * args.stage_iters
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "schedule": "Sec. 4.1 warm-up, 5 stages",
+                      "value": NW * wl.total * 5 * args.stage_iters / (total_ms * 1e-3),
+                      "config": {"workload": wl.name, "elements": wl.total,
+                                 "simulated_workers": NW, "stage_iters": args.stage_iters,
+                                 "streams": NS, "clip_threshold": wl.clip_threshold},
+                      "stages": rows}))
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle on the same metric and config (bounded sample per step)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -455,12 +532,17 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--warmup-schedule", action="store_true",
+                    help="run the 5-stage sparsity warm-up and report per-stage timings")
+    ap.add_argument("--stage-iters", type=int, default=20)
     ap.add_argument("--traffic", type=float, default=None,
                     help="DRAM bytes per launch of the dominant kernel from an ncu capture")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.warmup_schedule:
+        run_schedule(args)
     else:
         run_ours(args)
 
