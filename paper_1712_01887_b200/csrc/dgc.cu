@@ -44,11 +44,6 @@ int poisson_rank(double lambda, double eps) {
   return r + 1;
 }
 
-struct DevBuf {
-  void* ptr = nullptr;
-  size_t bytes = 0;
-};
-
 }  // namespace
 
 struct dgc_state {

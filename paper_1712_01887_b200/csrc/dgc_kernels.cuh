@@ -11,8 +11,11 @@
 //                      512-element segment, into their part's candidate list
 //   k_select           exact k-th largest |v'| among a tensor's candidates (radix
 //                      select on the IEEE bit pattern), tie quota, per-part output bases
+//   k_big_hist<0..2>,  the same selection for tensors whose candidates do not fit one block
+//   k_big_final        (warm-up sparsities, very large tensors): three histogram rounds
 //   k_emit_mask        Alg. 4 "G~ <- V (.) Mask", Sec. 3.3 masking: ordered (index, value)
-//                      pairs, then u = v = 0 at the sent entries
+//                      pairs; u = v = 0 at the sent entries, either at once or (low
+//                      sparsity) recorded as bits that the next call's kernels apply
 //
 // The sample only proposes; if a proposal lets fewer than k_j entries or more
 // than the list capacity through, that tensor is selected from the whole of v'
