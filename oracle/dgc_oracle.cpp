@@ -38,6 +38,7 @@
 #include <cmath>
 #include <cstdint>
 #include <cstring>
+#include <functional>
 #include <utility>
 #include <vector>
 
@@ -266,6 +267,125 @@ int64_t dgc_oracle_decode_runlength(const uint16_t* runs, const float* values, i
     pos += 1;
   }
   return count;
+}
+
+// ---------------------------------------------------------------------------------------
+// The sampled selection as Sec. 5 states it ("paper-literal" mode): the threshold is taken
+// from a sample and applied to the whole tensor; only "if the number of gradients exceeding
+// the threshold is far more than expected, a precise threshold is calculated from the
+// already-selected gradients".  The number of entries sent then varies.  Readings (the paper
+// gives none of these): the sample is one group of 4 consecutive elements per stratum at a
+// hashed position (below); thr is the k_s-th largest sampled |v|, k_s = ceil(S (1 - s)), so
+// that "|v| > thr" keeps n k_s / (S + 1) ~ n (1 - s) entries on average; "far more" = more
+// than 2 k_j, in which case the exact top-k_j is sent; tensors of <= 8192 elements are their
+// own sample, and for them thr is the (k_j + 1)-th largest |v| (the largest entry not to be
+// sent), so that "|v| > thr" keeps the top k_j minus whatever ties with thr.  The positions come from a counter-based hash that this
+// file and the CUDA library each implement.
+
+static inline uint64_t oracle_mix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+// Groups of 4 elements sampled from a tensor of n elements (0: the whole tensor is the sample).
+int64_t dgc_oracle_sample_groups(int64_t n, double sparsity, double sample_ratio) {
+  if (n <= 8192) return 0;
+  const double ratio = sample_ratio > 0.0 ? sample_ratio : 0.01;
+  long long G = (long long)std::ceil(ratio * (double)n / 4.0);
+  const long long enough = (long long)std::ceil(1024.0 / std::max(1.0 - sparsity, 1e-9) / 4.0);
+  G = std::min(G, enough);
+  G = std::max(G, 64LL);
+  G = std::min(G, std::min((long long)(n / 4), 16384LL));
+  return G;
+}
+
+// Selection of one tensor in paper-literal mode.  v: the n accumulated values (already
+// updated).  Returns the number of entries chosen; their local indices ascending in sel_idx
+// (capacity min(n, 2k)).
+int64_t dgc_oracle_select_sampled(int64_t n, const float* v, int64_t k, double sparsity,
+                                  double sample_ratio, uint64_t call_seed, int32_t tensor_index,
+                                  int64_t* sel_idx) {
+  const int64_t G = dgc_oracle_sample_groups(n, sparsity, sample_ratio);
+  std::vector<uint32_t> sample;
+  if (G == 0) {
+    sample.resize(static_cast<size_t>(n));
+    for (int64_t i = 0; i < n; ++i) sample[static_cast<size_t>(i)] = magnitude_key(v[i]);
+  } else {
+    const uint32_t W = static_cast<uint32_t>((n / 4) / G);        // groups per stratum
+    sample.reserve(static_cast<size_t>(4 * G));
+    for (int64_t st = 0; st < G; ++st) {
+      const uint32_t h = static_cast<uint32_t>(oracle_mix64(
+          call_seed ^ (static_cast<uint64_t>(static_cast<uint32_t>(tensor_index)) << 32) ^
+          static_cast<uint64_t>(static_cast<uint32_t>(st))));
+      const uint64_t grp = static_cast<uint64_t>(st) * W +
+                           ((static_cast<uint64_t>(h) * static_cast<uint64_t>(W)) >> 32);
+      for (int c = 0; c < 4; ++c) sample.push_back(magnitude_key(v[4 * grp + c]));
+    }
+  }
+  const int64_t S = static_cast<int64_t>(sample.size());
+  const int64_t ks = dgc_oracle_topk_count(S, sparsity);
+  // rank of thr in the sample: k_s for a true sample, k + 1 when the tensor is its own sample;
+  // no threshold at all if that rank does not exist (everything is to be sent)
+  const int64_t rank = G == 0 ? k + 1 : ks;
+  bool have_thr = rank <= S;
+  uint32_t thr = 0;
+  if (have_thr) {
+    std::nth_element(sample.begin(), sample.begin() + (rank - 1), sample.end(),
+                     std::greater<uint32_t>());
+    thr = sample[static_cast<size_t>(rank - 1)];
+  }
+  std::vector<int64_t> pass;
+  for (int64_t i = 0; i < n; ++i)
+    if (!have_thr || magnitude_key(v[i]) > thr) pass.push_back(i);
+  if (static_cast<int64_t>(pass.size()) > 2 * k) {
+    // far more than expected: the precise top-k_j (same order as everywhere: ties to the lower index)
+    dgc_oracle_select_topk(n, v, k, sel_idx, 0);
+    return k;
+  }
+  for (size_t r = 0; r < pass.size(); ++r) sel_idx[r] = pass[r];
+  return static_cast<int64_t>(pass.size());
+}
+
+// One iteration in paper-literal mode: clip, momentum correction, then per tensor the
+// sampled selection above, emission and masking.  The pairs of all tensors are packed back to
+// back (tensor order, ascending index); nnz_out[j] = entries sent from tensor j.
+// seed/iteration give call_seed = seed * 0x9E3779B97F4A7C15 + iteration (mod 2^64).
+int64_t dgc_oracle_compress_sampled(int32_t num_tensors, const int64_t* offset,
+                                    const int64_t* numel, const int64_t* k, float* u, float* v,
+                                    const float* g, float momentum, double clip_threshold,
+                                    int32_t num_workers, int32_t coef_override_flag,
+                                    float coef_override, int32_t nesterov, double sparsity,
+                                    double sample_ratio, uint64_t seed, int64_t iteration,
+                                    int32_t* out_idx, float* out_val, int64_t* nnz_out,
+                                    double* norm_out, float* coef_out) {
+  double norm = 0.0;
+  float coef = 1.0f;
+  dgc_oracle_clip_coef(num_tensors, offset, numel, g, clip_threshold, num_workers, &norm, &coef);
+  if (coef_override_flag) coef = coef_override;
+  *norm_out = norm;
+  *coef_out = coef;
+  dgc_oracle_momentum_correction(num_tensors, offset, numel, u, v, g, momentum, coef, nesterov);
+  const uint64_t call_seed = seed * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(iteration);
+  std::vector<int64_t> sel;
+  int64_t out = 0;
+  for (int32_t j = 0; j < num_tensors; ++j) {
+    const int64_t o = offset[j];
+    sel.assign(static_cast<size_t>(std::min(numel[j], 2 * k[j])), 0);
+    const int64_t c = dgc_oracle_select_sampled(numel[j], v + o, k[j], sparsity, sample_ratio,
+                                                call_seed, j, sel.data());
+    nnz_out[j] = c;
+    for (int64_t r = 0; r < c; ++r) {
+      const int64_t i = o + sel[static_cast<size_t>(r)];
+      out_idx[out] = static_cast<int32_t>(i);
+      out_val[out] = v[i];
+      ++out;
+      v[i] = 0.0f;
+      u[i] = 0.0f;
+    }
+  }
+  return out;
 }
 
 }  // extern "C"

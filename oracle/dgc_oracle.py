@@ -65,6 +65,14 @@ def lib() -> ctypes.CDLL:
                                                    ctypes.c_int64]
         L.dgc_oracle_apply_sgd.restype = None
         L.dgc_oracle_apply_sgd.argtypes = [_f32p, _f32p, ctypes.c_int64, ctypes.c_float]
+        L.dgc_oracle_sample_groups.restype = ctypes.c_int64
+        L.dgc_oracle_sample_groups.argtypes = [ctypes.c_int64, ctypes.c_double, ctypes.c_double]
+        L.dgc_oracle_compress_sampled.restype = ctypes.c_int64
+        L.dgc_oracle_compress_sampled.argtypes = [
+            ctypes.c_int32, _i64p, _i64p, _i64p, _f32p, _f32p, _f32p, ctypes.c_float,
+            ctypes.c_double, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
+            ctypes.c_double, ctypes.c_double, ctypes.c_uint64, ctypes.c_int64, _i32p, _f32p,
+            _i64p, _f64p, _f32p]
         L.dgc_oracle_encode_runlength.restype = ctypes.c_int64
         L.dgc_oracle_encode_runlength.argtypes = [_i32p, _f32p, ctypes.c_int64,
                                                   ctypes.POINTER(ctypes.c_uint16), _f32p,
@@ -174,6 +182,31 @@ class Worker:
             ctypes.byref(norm),
             ctypes.byref(coef))
         return CompressResult(idx, val, norm.value, np.float32(coef.value))
+
+
+def sample_groups(n: int, sparsity: float, sample_ratio: float = 0.01) -> int:
+    return int(lib().dgc_oracle_sample_groups(int(n), float(sparsity), float(sample_ratio)))
+
+
+def compress_sampled(worker: "Worker", g: np.ndarray, seed: int, iteration: int,
+                     sample_ratio: float = 0.01, coef_override=None):
+    """Paper-literal sampled selection (Sec. 5) on a Worker's state: returns
+    (CompressResult with the packed lists, nnz per tensor)."""
+    g = _chk(g, np.float32)
+    cap = int(np.minimum(worker.numel, 2 * worker.k).sum())
+    idx = np.empty(cap, dtype=np.int32)
+    val = np.empty(cap, dtype=np.float32)
+    nnz = np.zeros(len(worker.numel), dtype=np.int64)
+    norm = ctypes.c_double()
+    coef = ctypes.c_float()
+    n = lib().dgc_oracle_compress_sampled(
+        len(worker.numel), _p(worker.offset, _i64p), _p(worker.numel, _i64p), _p(worker.k, _i64p),
+        _p(worker.u, _f32p), _p(worker.v, _f32p), _p(g, _f32p), ctypes.c_float(worker.momentum),
+        worker.clip_threshold, worker.num_workers, int(coef_override is not None),
+        ctypes.c_float(0.0 if coef_override is None else float(coef_override)),
+        int(worker.nesterov), worker.sparsity, float(sample_ratio), int(seed), int(iteration),
+        _p(idx, _i32p), _p(val, _f32p), _p(nnz, _i64p), ctypes.byref(norm), ctypes.byref(coef))
+    return CompressResult(idx[:n].copy(), val[:n].copy(), norm.value, np.float32(coef.value)), nnz
 
 
 def decode_accumulate(idx_lists, val_lists, dense_len: int) -> np.ndarray:

@@ -458,3 +458,97 @@ def test_encode_runlength_round_trip_and_size():
     runs, values = O.encode_runlength(idx, np.ones(k, np.float32), k + 64)
     ratio = 4 * L / (6 * runs.size)
     assert 600 < ratio <= 4 / (6 * 0.001) + 1e-9
+
+
+# ------------------------------------------------------------------ paper-literal sampled selection (Sec. 5)
+
+def _numpy_topk_set(v, k):
+    return set(_numpy_topk(v, k).tolist())
+
+
+def test_sampled_selection_small_tensor_is_its_own_sample():
+    """n <= 8192: the sample is the tensor, thr is the (k+1)-th largest |v|, "|v| > thr" keeps
+    the top k minus whatever ties with thr: checked against numpy's sort."""
+    rng = np.random.default_rng(41)
+    for n, s in ((1000, 0.99), (8192, 0.999), (64, 0.75), (5, 0.0)):
+        w = O.Worker([0], [n], n, 1, 0.0, 0.0, s)
+        g = rng.standard_normal(n).astype(np.float32)
+        r, nnz = O.compress_sampled(w, g.copy(), seed=1, iteration=0)
+        k = O.topk_count(n, s)
+        if k == n:
+            expect = np.arange(n)
+        else:
+            a = np.abs(g)
+            thr = np.sort(a)[::-1][k]
+            expect = np.flatnonzero(a > thr)
+        assert r.idx.tolist() == expect.tolist() and nnz.tolist() == [expect.size]
+        assert r.val.tobytes() == g[expect].tobytes()
+    # ties with the (k+1)-th are not sent
+    w = O.Worker([0], [8], 8, 1, 0.0, 0.0, 0.75)      # k = 2
+    r, nnz = O.compress_sampled(w, _f32([5, 3, 3, 3, 1, 0, 0, 0]), seed=0, iteration=0)
+    assert r.idx.tolist() == [0] and nnz.tolist() == [1]
+
+
+def test_sampled_selection_threshold_is_a_sample_quantile():
+    """Large iid tensors: what passes is a superset or subset of the exact top-k with a count
+    near k (the sample holds k_s = 40 of the entries to send), every sent entry dominates every
+    unsent one, and nothing beyond 2k is ever sent."""
+    rng = np.random.default_rng(43)
+    n, s = 400000, 0.99
+    k = O.topk_count(n, s)
+    assert O.sample_groups(n, s) == 1000            # 1% of n / 4, below the other caps
+    counts = []
+    for it in range(6):
+        w = O.Worker([0], [n], n, 1, 0.0, 0.0, s)
+        g = rng.standard_normal(n).astype(np.float32)
+        r, nnz = O.compress_sampled(w, g.copy(), seed=7, iteration=it)
+        c = int(nnz[0])
+        counts.append(c)
+        assert 0.4 * k < c < 1.8 * k              # 40 of the 4000 sampled lie above thr: +-16 %
+        sent = np.zeros(n, bool)
+        sent[r.idx] = True
+        assert np.abs(g[sent]).min() > np.abs(g[~sent]).max()
+        top = _numpy_topk_set(g, k)
+        got = set(r.idx.tolist())
+        assert got <= top or top <= got
+        assert not w.u[r.idx].any() and not w.v[r.idx].any()
+    assert len(set(counts)) > 1                       # the count really varies with the sample
+
+
+def test_sampled_selection_far_more_than_expected_gives_exact_topk():
+    """n = 100000 at 99.9 %: 1000 sampled elements, k_s = 1, so thr is the sample maximum and
+    the number of entries above it is roughly exponential with mean k: more than 2k pass in
+    about one call in seven, and then exactly the top k must be sent."""
+    rng = np.random.default_rng(53)
+    n, s = 100000, 0.999
+    k = O.topk_count(n, s)
+    assert O.sample_groups(n, s) == 250
+    g = rng.standard_normal(n).astype(np.float32)
+    top = _numpy_topk(g, k)
+    kinds = set()
+    for it in range(60):
+        w = O.Worker([0], [n], n, 1, 0.0, 0.0, s)
+        r, nnz = O.compress_sampled(w, g.copy(), seed=5, iteration=it)
+        c = int(nnz[0])
+        assert c <= 2 * k
+        sent = np.zeros(n, bool)
+        sent[r.idx] = True
+        if c:
+            assert np.abs(g[sent]).min() > np.abs(g[~sent]).max()
+        if c == k:
+            assert r.idx.tolist() == top.tolist()
+        kinds.add("exact" if c == k else ("fewer" if c < k else "more"))
+    assert kinds == {"exact", "fewer", "more"}
+
+
+def test_sampled_selection_depends_on_seed_and_iteration_only_through_the_sample():
+    rng = np.random.default_rng(47)
+    n, s = 200000, 0.999
+    g = rng.standard_t(3, n).astype(np.float32)
+    outs = []
+    for seed, it in ((1, 0), (1, 0), (1, 1), (2, 0)):
+        w = O.Worker([0], [n], n, 1, 0.0, 0.0, s)
+        r, nnz = O.compress_sampled(w, g.copy(), seed=seed, iteration=it)
+        outs.append(r.idx.tolist())
+    assert outs[0] == outs[1]                          # deterministic
+    assert outs[0] != outs[2] or outs[0] != outs[3]    # another sample, another threshold
