@@ -478,6 +478,53 @@ def run_schedule(args):
                       "stages": rows}))
 
 
+def run_literal(args):
+    """Compress-only timing of the paper-literal sampled selection (select_mode = 1, Sec. 5 as
+    stated: variable number of entries, so the fixed-size step of the headline does not apply)."""
+    import torch
+    from paper_1712_01887_b200 import build
+    build.build()
+    from paper_1712_01887_b200 import binding as B
+    wl = I.workload(args.workload) if args.workload != "sweep" else I.workload("sweep", n=args.n)
+    if args.clip is not None:
+        wl.clip_threshold = args.clip
+    if args.sparsity is not None:
+        wl.sparsity = args.sparsity
+    NW = args.workers or wl.num_workers
+    off, L, hosts = _make_pool(wl, NW, 0)
+    res = {}
+    for mode in (0, 1):
+        states = [B.State(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold, wl.sparsity,
+                          sample_ratio=wl.sample_ratio, seed=I.BASE_SEED + w, select_mode=mode)
+                  for w in range(NW)]
+        pool = [[h.cuda() for h in row] for row in hosts]
+        cap = states[0].max_nnz
+        oi = [torch.empty(cap, dtype=torch.int32, device="cuda") for _ in range(NW)]
+        ov = [torch.empty(cap, dtype=torch.float32, device="cuda") for _ in range(NW)]
+        for t in range(args.warmup):
+            for w in range(NW):
+                states[w].compress(pool[w][t % POOL], oi[w], ov[w])
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(args.steps):
+            for w in range(NW):
+                states[w].compress(pool[w][t % POOL], oi[w], ov[w])
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / (args.steps * NW)
+        total, per = states[0].nnz()
+        res["exact" if mode == 0 else "paper_literal"] = {
+            "compress_ms": ms, "elements_per_s": wl.total / (ms * 1e-3),
+            "entries_sent_last_call": total, "sum_k": int(states[0].k.sum())}
+        for st in states:
+            st.close()
+        del pool
+    print(json.dumps({"metric": METRIC, "unit": UNIT, "config": {"workload": wl.name,
+                      "elements": wl.total, "sparsity": wl.sparsity, "simulated_workers": NW},
+                      "select_modes": res}))
+
+
 def run_reference(args):
     """--impl reference: the CPU oracle on the same metric and config (bounded sample per step)."""
     rank = int(os.environ.get("RANK", "0"))
@@ -532,6 +579,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    ap.add_argument("--compare-select-modes", action="store_true",
+                    help="compress-only timing of exact vs paper-literal sampled selection")
     ap.add_argument("--warmup-schedule", action="store_true",
                     help="run the 5-stage sparsity warm-up and report per-stage timings")
     ap.add_argument("--stage-iters", type=int, default=20)
@@ -543,6 +592,8 @@ def main():
         run_reference(args)
     elif args.warmup_schedule:
         run_schedule(args)
+    elif args.compare_select_modes:
+        run_literal(args)
     else:
         run_ours(args)
 

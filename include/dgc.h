@@ -68,7 +68,10 @@ typedef struct dgc_config {
                                      sample maximum, which forces the full-selection path)     */
   int32_t        nesterov;        /* 0: Algorithm 4 (vanilla momentum, Eq. 5).  1: Algorithm 5
                                      (Appendix B): U <- m*(U + g) ; V <- (V + U) + g           */
-  int32_t        reserved;        /* set to 0                                                   */
+  int32_t        select_mode;     /* 0: exact top-k_j per tensor (the sample only proposes).
+                                     1: Sec. 5 as stated ("paper-literal"): the threshold comes
+                                     from the sample, |v| > thr is sent, at most 2 k_j entries
+                                     per tensor; the count varies, see dgc_get_nnz             */
 } dgc_config;
 
 typedef struct dgc_status {
@@ -232,6 +235,18 @@ int64_t dgc_runlength_workspace_bytes(int64_t entries);
 
 /* Synchronises `stream`, then reports counters of the last dgc_compress. */
 int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out);
+
+/* Entries the last dgc_compress wrote, in total and per tensor (host outputs, either may be
+ * NULL).  select_mode 0: the fixed k_j, no synchronisation.  select_mode 1 (Sec. 5 taken
+ * literally): synchronises `stream` and reads the counts.  In that mode the threshold of
+ * tensor j is the k_s-th largest |v| of its sample (k_s = ceil(S (1 - s)), S sampled
+ * elements: one group of 4 per stratum at a hashed position; tensors of <= 8192 elements are
+ * their own sample and use their (k_j + 1)-th largest |v|); every entry with |v| > thr is
+ * sent, unless more than 2 k_j pass ("far more than expected"), in which case the exact
+ * top-k_j is sent.  The tensors' lists are packed back to back in tensor order (ascending
+ * index overall); dgc_max_nnz() is then the capacity bound sum_j min(n_j, 2 k_j), and the
+ * out_offset of dgc_layout is not used. */
+int32_t dgc_get_nnz(dgc_state* st, void* stream, int64_t* total_out, int64_t* per_tensor);
 
 /* Synchronises `stream`, then copies per-tensor results of the last
  * dgc_compress to host arrays [num_tensors] (either may be NULL):

@@ -36,7 +36,7 @@ class Config(ctypes.Structure):
                 ("clip_threshold", ctypes.c_float), ("sparsity", ctypes.c_double),
                 ("sample_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
                 ("device", ctypes.c_int32), ("debug_sample_rank", ctypes.c_int32),
-                ("nesterov", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("nesterov", ctypes.c_int32), ("select_mode", ctypes.c_int32)]
 
 
 class Status(ctypes.Structure):
@@ -73,6 +73,7 @@ _sigs = {
                                               ctypes.c_int64, _vp]),
     "dgc_runlength_max_entries": (ctypes.c_int64, [ctypes.c_int64, ctypes.c_int64]),
     "dgc_runlength_workspace_bytes": (ctypes.c_int64, [ctypes.c_int64]),
+    "dgc_get_nnz": (ctypes.c_int32, [_vp, _vp, _i64p, _i64p]),
     "dgc_get_status": (ctypes.c_int32, [_vp, _vp, ctypes.POINTER(Status)]),
     "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
@@ -132,11 +133,11 @@ class State:
     def __init__(self, tensor_numel: Sequence[int], num_workers: int, momentum: float,
                  clip_threshold: float, sparsity: float, sample_ratio: float = 0.01,
                  seed: int = 0, device: int = 0, debug_sample_rank: int = 0,
-                 nesterov: bool = False):
+                 nesterov: bool = False, select_mode: int = 0):
         numel = (ctypes.c_int64 * len(tensor_numel))(*[int(n) for n in tensor_numel])
         cfg = Config(len(tensor_numel), int(num_workers), numel, float(momentum),
                      float(clip_threshold), float(sparsity), float(sample_ratio), int(seed),
-                     int(device), int(debug_sample_rank), int(bool(nesterov)), 0)
+                     int(device), int(debug_sample_rank), int(bool(nesterov)), int(select_mode))
         self._h = _vp()
         self.num_tensors = len(tensor_numel)
         self.device = int(device)
@@ -194,6 +195,14 @@ class State:
         s = Status()
         _check(_lib.dgc_get_status(self._h, _stream(stream), ctypes.byref(s)), "dgc_get_status")
         return s
+
+    def nnz(self, stream=None):
+        """(total, per-tensor) entries written by the last compress call."""
+        total = ctypes.c_int64()
+        per = np.zeros(self.num_tensors, np.int64)
+        _check(_lib.dgc_get_nnz(self._h, _stream(stream), ctypes.byref(total),
+                                per.ctypes.data_as(_i64p)), "dgc_get_nnz")
+        return int(total.value), per
 
     def thresholds(self, stream=None):
         kth = np.zeros(self.num_tensors, np.uint32)

@@ -135,6 +135,7 @@ void build_host_plan(dgc_state* st, double sparsity) {
   st->big_parts.clear();
   st->big_tensors.clear();
   const int key_cap = select_key_cap(st);
+  const bool literal = st->cfg.select_mode == 1;
   int64_t pos = 0, out = 0, cbase = 0;
   st->max_tensor_expect = 0;
   for (int j = 0; j < T; ++j) {
@@ -145,7 +146,7 @@ void build_host_plan(dgc_state* st, double sparsity) {
     t.end = (int32_t)(pos + n);
     t.k = (int32_t)k;
     t.out_off = (int32_t)out;
-    out += k;
+    out += literal ? std::min<int64_t>(n, 2 * k) : k;   // literal: capacity, the count varies
     const int64_t nseg = (n + kSeg - 1) / kSeg;
     const int64_t nparts = (nseg + kPartSegs - 1) / kPartSegs;
     // sampling plan
@@ -166,7 +167,14 @@ void build_host_plan(dgc_state* st, double sparsity) {
       const double lambda = S * (double)k / (double)n;
       rank = poisson_rank(lambda, 1e-9) + 2;
       if (st->cfg.debug_sample_rank > 0) rank = st->cfg.debug_sample_rank;
-      if (rank >= S / 2) {
+      if (literal) {
+        // Sec. 5 as stated: thr = the sample's k_s-th largest key, k_s = ceil(S (1 - s)); about
+        // k entries pass, at most 2k are sent, anything beyond overflows into the exact path
+        rank = (int)topk_count((int64_t)S, sparsity);
+        groups = (int)G;
+        cap_total = std::min((double)n, 2.0 * (double)k + 1024.0);
+        expect_keys = cap_total;
+      } else if (rank >= S / 2) {
         sampled = false;
       } else {
         groups = (int)G;
@@ -199,6 +207,8 @@ void build_host_plan(dgc_state* st, double sparsity) {
       if (sampled) {
         const int64_t share = (int64_t)std::ceil(cap_total / (double)nparts);
         cap = std::min<int64_t>(elems, std::max<int64_t>(4 * share, 8192));
+        // paper-literal: a part may only overflow when more than 2k entries passed in all
+        if (literal) cap = std::min<int64_t>(elems, std::max<int64_t>(cap, 2 * k + 1));
       }
       PartMeta m{};
       m.tensor = j;
@@ -237,6 +247,7 @@ int32_t upload_plan(dgc_state* st, bool first) {
   const size_t o_pthr = o; o = up16(o + P * 4);
   const size_t o_kth = o; o = up16(o + T * 4);
   const size_t o_cand = o; o = up16(o + T * 4);
+  const size_t o_nnz = o; o = up16(o + T * 4);
   const size_t o_seg = o; o = up16(o + S * 4);
   const size_t o_samp = o; o = up16(o + NS * sizeof(SampleBlock));
   const size_t o_skeys = o; o = up16(o + (size_t)st->sample_keys_total * 4);
@@ -274,6 +285,8 @@ int32_t upload_plan(dgc_state* st, bool first) {
   p.p_thr = (uint32_t*)(d + o_pthr);
   p.t_kth = (uint32_t*)(d + o_kth);
   p.t_cand = (int32_t*)(d + o_cand);
+  p.t_nnz = (int32_t*)(d + o_nnz);
+  p.literal = st->cfg.select_mode == 1 ? 1 : 0;
   p.seg_part = (const int32_t*)(d + o_seg);
   p.sample_blocks = (const SampleBlock*)(d + o_samp);
   p.sample_keys = (uint32_t*)(d + o_skeys);
@@ -371,6 +384,7 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   *out = nullptr;
   if (cfg->num_tensors < 1 || !cfg->tensor_numel || cfg->num_workers < 1) return DGC_EINVAL;
   if (!(cfg->sparsity >= 0.0 && cfg->sparsity < 1.0)) return DGC_EINVAL;
+  if (cfg->select_mode != 0 && cfg->select_mode != 1) return DGC_EINVAL;
   if (!(cfg->sample_ratio >= 0.0 && cfg->sample_ratio <= 0.5)) return DGC_EINVAL;
   if (!(cfg->momentum == cfg->momentum)) return DGC_EINVAL;
   int64_t padded = 0;
@@ -775,6 +789,26 @@ int32_t dgc_profile_read(dgc_state* st, float* ms_out, int32_t capacity, int32_t
                                     st->prof_ev[6 * i + k + 1]));
   }
   *count_out = n;
+  return DGC_OK;
+}
+
+int32_t dgc_get_nnz(dgc_state* st, void* stream, int64_t* total_out, int64_t* per_tensor) {
+  if (!st || !st->alive) return DGC_ESTATE;
+  const size_t T = st->cfg.num_tensors;
+  std::vector<int32_t> h(T);
+  if (st->cfg.select_mode == 1) {
+    DGC_CUDA(cudaStreamSynchronize(as_stream(stream)));
+    if (st->iterations == 0) std::fill(h.begin(), h.end(), 0);
+    else DGC_CUDA(cudaMemcpy(h.data(), st->plan.t_nnz, T * 4, cudaMemcpyDeviceToHost));
+  } else {
+    for (size_t j = 0; j < T; ++j) h[j] = st->tm[j].k;
+  }
+  int64_t total = 0;
+  for (size_t j = 0; j < T; ++j) {
+    if (per_tensor) per_tensor[j] = h[j];
+    total += h[j];
+  }
+  if (total_out) *total_out = total;
   return DGC_OK;
 }
 

@@ -62,6 +62,7 @@ constexpr int kBigLastBins = 512;
 constexpr int kBigLastStride = 516;    // 513 suffix sums, padded to a multiple of 4 words
 constexpr int kBigStateWords = 64;
 constexpr int kBigNear = 64;           // round-0 digits this close above the proposal's get private bins
+constexpr int kTakeAllTies = 0x3FFFFFFF;   // tie quota meaning "every entry tied with the threshold"
 constexpr int kDecodeTile = 4096;
 constexpr int kDecodeThreads = 256;
 
@@ -94,6 +95,8 @@ struct Plan {
   PartSel* psel;
   int32_t* p_count;          // candidates appended per part (reset by k_emit_mask)
   uint32_t* p_thr;           // proposed threshold per part (0 for tensors that are not sampled)
+  int32_t* t_nnz;            // per tensor: entries sent by the last call (paper-literal mode)
+  int32_t literal;           // 1: paper-literal sampled selection (Sec. 5), variable count
   uint32_t* t_kth;           // per tensor: threshold of the last call (reporting)
   int32_t* t_cand;           // per tensor: candidates of the last call, -1 = full selection
   const int32_t* seg_part;   // part of every segment
@@ -502,8 +505,9 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
         },
         rank, 0u, kmax, hist, sh, n_gt);
   }
-  // a proposal of 0 would let every entry through: insist on non-zero magnitude
-  const uint32_t thr = kth > 1u ? kth : 1u;
+  // exact mode: a proposal of 0 would let every entry through, so insist on non-zero
+  // magnitude.  Paper-literal mode: the mask is "|v| > thr" with thr the sample's rank-k_s key.
+  const uint32_t thr = p.literal ? kth + 1u : (kth > 1u ? kth : 1u);
   for (int q = tid; q < t.part_num; q += kSampleThreads) p.p_thr[t.part_first + q] = thr;
 }
 
@@ -690,7 +694,16 @@ k_select(Plan p, int smem_keys, int parity) {
     __syncthreads();
   }
   const bool overflow = s_flag != 0;
-  if (overflow || total < k) {
+  // Paper-literal mode (Sec. 5): what passed the sampled threshold is sent as it is unless it
+  // is "far more than expected" (more than 2k: then the precise top-k); a tensor that is its
+  // own sample (not sampled: every entry is a candidate) sends what exceeds its (k+1)-th key.
+  const bool literal = p.literal != 0;
+  const bool lit_sampled_all = literal && t.groups > 0 && !overflow && total <= 2 * k;
+  const bool lit_own = literal && t.groups == 0;
+  const bool lit_own_all = lit_own && k + 1 > total;
+  const int rank = lit_own ? k + 1 : k;
+  if (overflow || (!literal && total < k)) {
+    if (tid == 0) p.t_nnz[j] = k;
     // full-selection path: k_emit_mask's block of the tensor's first part does it
     for (int q = tid; q < pn; q += kSelectThreads) {
       PartSel ps;
@@ -733,7 +746,13 @@ k_select(Plan p, int smem_keys, int parity) {
   }
   int n_gt;
   uint32_t kth;
-  if (in_smem) {
+  if (lit_sampled_all) {
+    kth = __ldcg(p.p_thr + p0) - 1u;             // every candidate exceeds it (p_thr >= 1 here)
+    n_gt = total;
+  } else if (lit_own_all) {
+    kth = 0u;                                    // k = n: everything, zeros included
+    n_gt = 0;
+  } else if (in_smem) {
     const int iters = (total + kSelectThreads - 1) / kSelectThreads;
     kth = block_select_desc(
         [&](auto f) {
@@ -743,7 +762,7 @@ k_select(Plan p, int smem_keys, int parity) {
             f(valid, valid ? skeys[i] : kbase);
           }
         },
-        k, kbase, kmax, hist, sh, n_gt);
+        rank, kbase, kmax, hist, sh, n_gt);
   } else {
     kth = block_select_desc(
         [&](auto f) {
@@ -758,10 +777,12 @@ k_select(Plan p, int smem_keys, int parity) {
             }
           }
         },
-        k, kbase, kmax, hist, sh, n_gt);
+        rank, kbase, kmax, hist, sh, n_gt);
   }
-  const int quota = k - n_gt;   // ties (|v'| == kth) to take, lowest indices first
-  const int out_off = t.out_off;
+  // ties (|v'| == kth) to take, lowest indices first
+  const int quota = lit_sampled_all ? 0 : lit_own_all ? kTakeAllTies : lit_own ? 0 : k - n_gt;
+  const int nnz = lit_sampled_all ? total : lit_own_all ? total : lit_own ? n_gt : k;
+  const int out_off = literal ? 0 : t.out_off;   // paper-literal: k_emit_mask adds the tensor's base
   if (tables) {
     // per part: strictly-greater and tied candidates (a single part needs no count: it takes
     // the whole quota and k_emit_mask stops at the quota by itself)
@@ -859,6 +880,7 @@ k_select(Plan p, int smem_keys, int parity) {
   if (tid == 0) {
     p.t_kth[j] = kth;
     p.t_cand[j] = total;
+    p.t_nnz[j] = nnz;
     atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
   }
 }
@@ -1026,10 +1048,30 @@ k_big_final(Plan p, int parity) {
   int ex, exo, total, overflow;
   block_excl_scan2(mine, over, sh, ex, exo, total, overflow);
   __syncthreads();
-  const bool dense = overflow != 0 || total < k;
+  const bool literal = p.literal != 0;
+  const bool dense = overflow != 0 || (!literal && total < k);
+  // paper-literal mode: at most 2k passed the sampled threshold -> all of them are sent
+  const bool all_pass = literal && !dense && total <= 2 * k;
+  const int out_off = literal ? 0 : t.out_off;
   uint32_t kth = 0;
   int quota = 0;
-  if (!dense) {
+  if (all_pass) {
+    kth = __ldcg(p.p_thr + p0) - 1u;            // every candidate exceeds it
+    int run = 0;
+    for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+      const int q = q0 + tid;
+      const int c = q < pn ? __ldcg(p.p_count + p0 + q) : 0;
+      int ex, e2, tot, t2;
+      block_excl_scan2(c, 0, sh, ex, e2, tot, t2);
+      if (q < pn) {
+        PartSel ps;
+        ps.kth = kth; ps.quota = 0; ps.out_base = out_off + run + ex; ps.dense = 0;
+        p.psel[p0 + q] = ps;
+      }
+      run += tot;
+      __syncthreads();
+    }
+  } else if (!dense) {
     const uint32_t prefix = (uint32_t)__ldcg(state + 32);
     const int rem2 = __ldcg(state + 33);
     int above;
@@ -1059,7 +1101,7 @@ k_big_final(Plan p, int parity) {
         PartSel ps;
         ps.kth = kth;
         ps.quota = max(0, min(quota - be, eq));
-        ps.out_base = t.out_off + bg + min(be, quota);
+        ps.out_base = out_off + bg + min(be, quota);
         ps.dense = 0;
         p.psel[p0 + q0 + tid] = ps;
       }
@@ -1088,6 +1130,7 @@ k_big_final(Plan p, int parity) {
       p.t_cand[j] = total;
       atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
     }
+    p.t_nnz[j] = all_pass ? total : k;
   }
 }
 
@@ -1102,8 +1145,8 @@ k_big_final(Plan p, int parity) {
 // Full-selection path (dense flag set by k_select): the block of the tensor's
 // first part selects from the whole of v' (radix select over global memory) and
 // emits by walking the tensor in order.  Same result; slow; rare.
-__device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int32_t* out_idx,
-                                  float* out_val, uint32_t* hist, int* sh) {
+__device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int out_first,
+                                  int32_t* out_idx, float* out_val, uint32_t* hist, int* sh) {
   const int tid = threadIdx.x, nt = blockDim.x;
   const int off = t.off;
   const int n = t.end - off;
@@ -1135,7 +1178,7 @@ __device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int
     int bg, be, tg, te;
     block_excl_scan2(gt, eq, sh, bg, be, tg, te);
     be += run_eq;
-    int pos = t.out_off + run_w + bg + (min(be, quota) - min(run_eq, quota));
+    int pos = out_first + run_w + bg + (min(be, quota) - min(run_eq, quota));
     int eqr = be;
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
@@ -1173,8 +1216,23 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   const int tid = threadIdx.x;
   // one round of independent loads: part record, selection result, candidate count
   const PartMeta pm = load_record(p.pm + part);
-  const PartSel ps = load_record(p.psel + part);
+  PartSel ps = load_record(p.psel + part);
   const int count = __ldcg(p.p_count + part);
+  int tensor_first = 0;      // first output slot of the tensor
+  if (p.literal) {
+    // paper-literal mode: the counts vary, so the tensors' lists are packed back to back:
+    // this tensor starts after what the earlier tensors send
+    __shared__ int s_first;
+    if (tid == 0) s_first = 0;
+    __syncthreads();
+    int mine = 0;
+    for (int q = tid; q < pm.tensor; q += kEmitThreads) mine += __ldcg(p.t_nnz + q);
+    mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+    if ((tid & 31) == 0 && mine) atomicAdd(&s_first, mine);
+    __syncthreads();
+    tensor_first = s_first;
+    ps.out_base += tensor_first;
+  }
   if (ps.dense) {
     __syncthreads();
     if (tid == 0) p.p_count[part] = 0;
@@ -1186,7 +1244,8 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
     }
     if (pm.first) {
       const TensorMeta t = load_record(p.tm + pm.tensor);
-      dense_select_emit(p, t, pm.tensor, out_idx, out_val, smask, sh);
+      dense_select_emit(p, t, pm.tensor, p.literal ? tensor_first : t.out_off, out_idx, out_val,
+                        smask, sh);
     }
     return;
   }

@@ -469,3 +469,50 @@ def test_deferred_masking_without_reading_state_between_iterations(P, sparsity):
         g[o:o + n] = rng.standard_normal(n).astype(np.float32)
     pair.step(g, rep, check_state=True)
     pair.close()
+
+
+@pytest.mark.parametrize("sparsity,numel,iters", [
+    (0.999, [100000, 8192, 64, 70001, 600000, 1 << 21], 12),
+    (0.99, [1 << 22, 300000, 5000, 9000], 4),           # the 2^22 tensor takes the multi-block path
+    (0.75, [200000, 1000], 3),
+])
+def test_paper_literal_sampled_selection_matches_oracle(P, sparsity, numel, iters):
+    """select_mode = 1: Sec. 5 as stated (threshold from the sample, variable count).  The
+    oracle draws the same sample (same counter-based hash); indices, values, per-tensor counts
+    and state must agree bit for bit, over several iterations and all three outcomes (fewer
+    than k, more than k, more than 2k -> exact top-k)."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    seed = 77
+    st = B.State(numel, 4, 0.9, 1.0, sparsity, seed=seed, select_mode=1)
+    L, off = st.arena_len, st.arena_offset
+    cpu = O.Worker(off, numel, L, 4, 0.9, 1.0, sparsity)
+    assert st.max_nnz == int(np.minimum(np.asarray(numel), 2 * cpu.k).sum())
+    oi = torch.empty(st.max_nnz, dtype=torch.int32, device="cuda")
+    ov = torch.empty(st.max_nnz, dtype=torch.float32, device="cuda")
+    rng = np.random.default_rng(3)
+    kinds = set()
+    for t in range(iters):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for o, n in zip(off, numel):
+            g[o:o + n] = rng.standard_normal(n).astype(np.float32)
+        st.compress(torch.from_numpy(g).cuda(), oi, ov)
+        status = st.status()
+        total, per = st.nnz()
+        snap = (cpu.u.copy(), cpu.v.copy())
+        r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t)
+        if np.float32(status.clip_coef).tobytes() != np.float32(r.coef).tobytes():
+            cpu.u[:], cpu.v[:] = snap
+            r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t,
+                                        coef_override=status.clip_coef)
+        assert per.tolist() == nnz.tolist(), (t, per, nnz)
+        assert total == r.idx.size
+        assert oi[:total].cpu().numpy().tobytes() == r.idx.tobytes()
+        assert ov[:total].cpu().numpy().tobytes() == r.val.tobytes()
+        u, v = st.read()
+        assert u.tobytes() == cpu.u.tobytes() and v.tobytes() == cpu.v.tobytes()
+        for c, k in zip(nnz, cpu.k):
+            kinds.add("k" if c == k else ("fewer" if c < k else "more"))
+    if sparsity == 0.999:
+        assert {"fewer", "more"} <= kinds
+    st.close()
