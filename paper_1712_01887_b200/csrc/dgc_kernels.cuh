@@ -224,12 +224,14 @@ __device__ __forceinline__ void block_excl_scan2(int a, int b, int* sh, int& ea,
 __host__ __device__ constexpr int kHistCopies(int threads) { return threads / 32 < 16 ? threads / 32 : 16; }
 __host__ __device__ constexpr int kHistWords(int threads) { return kHistCopies(threads) * 257 + 512; }
 
-template <class ForEach>
+template <int THREADS, class ForEach>
 __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank, uint32_t base,
                                                       uint32_t maxkey, uint32_t* hist, int* sh,
                                                       int& n_gt) {
-  const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31;
-  const int copies = kHistCopies(nt);
+  // THREADS = blockDim.x, a compile-time constant so that the slicing below costs no divisions
+  constexpr int nt = THREADS;
+  const int tid = threadIdx.x, lane = tid & 31;
+  constexpr int copies = kHistCopies(nt);
   uint32_t* mine = hist + ((tid >> 5) % copies) * 257;
   uint32_t* folded = hist + copies * 257;
   const uint32_t span = maxkey - base;
@@ -247,7 +249,8 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
     __syncthreads();
     {
       // fold (and clear) the private copies: thread t takes bin t & 255 of a slice of them
-      const int bin = tid & 255, groups = nt >> 8, grp = tid >> 8;
+      constexpr int groups = nt >> 8;
+      const int bin = tid & 255, grp = tid >> 8;
       const int c0 = grp * copies / groups, c1 = (grp + 1) * copies / groups;
       uint32_t t = 0;
       for (int c = c0; c < c1; ++c) {
@@ -451,7 +454,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
   bool done = false;
   if (rank <= owners) {
     // lower bound: rank-th largest of the thread maxima
-    const uint32_t low = block_select_desc([&](auto f) { f(tid < owners, tmax); }, rank, 0u, kmax,
+    const uint32_t low = block_select_desc<kSampleThreads>([&](auto f) { f(tid < owners, tmax); }, rank, 0u, kmax,
                                            hist, sh, n_gt);
     // keep the keys that reach it
 #pragma unroll 4
@@ -479,7 +482,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
     const int ns = s_cnt;
     if (ns <= kSampleSurvivors) {
       const int it2 = (ns + kSampleThreads - 1) / kSampleThreads;
-      kth = block_select_desc(
+      kth = block_select_desc<kSampleThreads>(
           [&](auto f) {
             for (int it = 0; it < it2; ++it) {
               const int i = it * kSampleThreads + tid;
@@ -491,7 +494,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
     }
   }
   if (!done) {
-    kth = block_select_desc(
+    kth = block_select_desc<kSampleThreads>(
         [&](auto f) {
           for (int it = 0; it < iters; ++it) {
             const int i = it * kSampleThreads + tid;
@@ -754,7 +757,7 @@ k_select(Plan p, int smem_keys, int parity) {
     n_gt = 0;
   } else if (in_smem) {
     const int iters = (total + kSelectThreads - 1) / kSelectThreads;
-    kth = block_select_desc(
+    kth = block_select_desc<kSelectThreads>(
         [&](auto f) {
           for (int it = 0; it < iters; ++it) {
             const int i = it * kSelectThreads + tid;
@@ -764,7 +767,7 @@ k_select(Plan p, int smem_keys, int parity) {
         },
         rank, kbase, kmax, hist, sh, n_gt);
   } else {
-    kth = block_select_desc(
+    kth = block_select_desc<kSelectThreads>(
         [&](auto f) {
           for (int q = 0; q < pn; ++q) {
             const int c = __ldcg(p.p_count + p0 + q);
@@ -1154,7 +1157,7 @@ __device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int
   const float* v = p.v + off;
   const int iters = (n + nt - 1) / nt;
   int n_gt;
-  const uint32_t kth = block_select_desc(
+  const uint32_t kth = block_select_desc<kEmitThreads>(
       [&](auto f) {
         for (int it = 0; it < iters; ++it) {
           const int i = it * nt + tid;
