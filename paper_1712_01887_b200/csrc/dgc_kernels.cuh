@@ -224,7 +224,9 @@ __device__ __forceinline__ void block_excl_scan2(int a, int b, int* sh, int& ea,
 __host__ __device__ constexpr int kHistCopies(int threads) { return threads / 32 < 16 ? threads / 32 : 16; }
 __host__ __device__ constexpr int kHistWords(int threads) { return kHistCopies(threads) * 257 + 512; }
 
-template <int THREADS, class ForEach>
+// PRIVATE = false skips the private copies (and the fold with its barrier): for a handful of
+// keys per block the atomics hardly collide and the fixed cost per pass is what counts.
+template <int THREADS, bool PRIVATE = true, class ForEach>
 __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank, uint32_t base,
                                                       uint32_t maxkey, uint32_t* hist, int* sh,
                                                       int& n_gt) {
@@ -238,16 +240,21 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
   const int passes = span == 0 ? 0 : (32 - __clz(span) + 7) / 8;
   uint32_t prefix = 0, mask = 0;
   int remaining = rank;
-  for (int i = tid; i < copies * 257 + 512; i += nt) hist[i] = 0;
+  if (PRIVATE) {
+    for (int i = tid; i < copies * 257 + 512; i += nt) hist[i] = 0;
+  } else {
+    for (int i = tid; i < 512; i += nt) folded[i] = 0;
+  }
   __syncthreads();
   int cur = 0;
   for (int shift = 8 * (passes - 1); shift >= 0; shift -= 8, cur ^= 1) {
+    uint32_t* target = PRIVATE ? mine : folded + cur * 256;
     for_each([&](bool valid, uint32_t key) {
       key -= base;
-      if (valid && (key & mask) == prefix) atomicAdd(&mine[(key >> shift) & 255u], 1u);
+      if (valid && (key & mask) == prefix) atomicAdd(&target[(key >> shift) & 255u], 1u);
     });
     __syncthreads();
-    {
+    if (PRIVATE) {
       // fold (and clear) the private copies: thread t takes bin t & 255 of a slice of them
       constexpr int groups = nt >> 8;
       const int bin = tid & 255, grp = tid >> 8;
@@ -258,8 +265,8 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
         hist[c * 257 + bin] = 0;
       }
       if (t) atomicAdd(&folded[cur * 256 + bin], t);
+      __syncthreads();
     }
-    __syncthreads();
     if (tid < 32) {
       const uint32_t* h = folded + cur * 256;
       const int hi = 255 - 8 * lane;          // this lane covers bins hi, hi-1, .., hi-7
@@ -454,7 +461,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
   bool done = false;
   if (rank <= owners) {
     // lower bound: rank-th largest of the thread maxima
-    const uint32_t low = block_select_desc<kSampleThreads>([&](auto f) { f(tid < owners, tmax); }, rank, 0u, kmax,
+    const uint32_t low = block_select_desc<kSampleThreads, false>([&](auto f) { f(tid < owners, tmax); }, rank, 0u, kmax,
                                            hist, sh, n_gt);
     // keep the keys that reach it
 #pragma unroll 4
@@ -482,7 +489,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_s
     const int ns = s_cnt;
     if (ns <= kSampleSurvivors) {
       const int it2 = (ns + kSampleThreads - 1) / kSampleThreads;
-      kth = block_select_desc<kSampleThreads>(
+      kth = block_select_desc<kSampleThreads, false>(
           [&](auto f) {
             for (int it = 0; it < it2; ++it) {
               const int i = it * kSampleThreads + tid;
@@ -757,15 +764,18 @@ k_select(Plan p, int smem_keys, int parity) {
     n_gt = 0;
   } else if (in_smem) {
     const int iters = (total + kSelectThreads - 1) / kSelectThreads;
-    kth = block_select_desc<kSelectThreads>(
-        [&](auto f) {
-          for (int it = 0; it < iters; ++it) {
-            const int i = it * kSelectThreads + tid;
-            const bool valid = i < total;
-            f(valid, valid ? skeys[i] : kbase);
-          }
-        },
-        rank, kbase, kmax, hist, sh, n_gt);
+    auto each = [&](auto f) {
+      for (int it = 0; it < iters; ++it) {
+        const int i = it * kSelectThreads + tid;
+        const bool valid = i < total;
+        f(valid, valid ? skeys[i] : kbase);
+      }
+    };
+    // up to two keys per thread: not worth private histograms
+    if (total <= 2 * kSelectThreads)
+      kth = block_select_desc<kSelectThreads, false>(each, rank, kbase, kmax, hist, sh, n_gt);
+    else
+      kth = block_select_desc<kSelectThreads, true>(each, rank, kbase, kmax, hist, sh, n_gt);
   } else {
     kth = block_select_desc<kSelectThreads>(
         [&](auto f) {
