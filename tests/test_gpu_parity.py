@@ -516,3 +516,21 @@ def test_paper_literal_sampled_selection_matches_oracle(P, sparsity, numel, iter
     if sparsity == 0.999:
         assert {"fewer", "more"} <= kinds
     st.close()
+
+
+def test_sparsity_lowered_after_creation_reallocates_scratch(P):
+    """dgc_set_sparsity towards a lower sparsity needs larger candidate lists than the state
+    was created with (and switches between immediate and deferred masking)."""
+    numel = [400000, 70001, 2000]
+    pair = P.Pair(numel, 2, 0.9, 1.0, 0.9999, seed=5)
+    rep = P.ParityReport()
+    rng = np.random.default_rng(29)
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    for s in (0.9999, 0.99, 0.5, 0.999, 0.0, 0.9):
+        pair.set_sparsity(s)
+        for t in range(2):
+            g = P.arena_with_padding_poison(L, off, numel)
+            for o, n in zip(off, numel):
+                g[o:o + n] = rng.standard_normal(n).astype(np.float32)
+            pair.step(g, rep, check_state=(t == 1))
+    pair.close()
