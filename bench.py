@@ -574,7 +574,7 @@ def main():
     ap.add_argument("--workers", type=int, default=None, help="simulated workers (default: config)")
     ap.add_argument("--clip", type=float, default=None, help="override thr_G (0 = off)")
     ap.add_argument("--sparsity", type=float, default=None)
-    ap.add_argument("--streams", type=int, default=4, help="streams the workers' compress calls use")
+    ap.add_argument("--streams", type=int, default=8, help="streams the workers' compress calls use")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
