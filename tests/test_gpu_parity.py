@@ -384,14 +384,14 @@ def test_runlength_of_compressed_resnet50_gradient(P):
     st.close()
 
 
-def test_workers_on_four_streams_like_the_benchmark(P):
-    """bench.py issues the simulated workers' compress calls round robin on four CUDA streams
+def test_workers_on_their_own_streams_like_the_benchmark(P):
+    """bench.py issues the simulated workers' compress calls on one CUDA stream per worker
     and joins them before the decode.  Same launch configuration here, on the ResNet-50-shaped
     set with all 8 workers: every worker must still match its oracle bit for bit."""
     from oracle import dgc_oracle as O
     from paper_1712_01887_b200 import binding as B
     wl = I.workload("resnet50")
-    NW, NS, T = 8, 4, 2
+    NW, NS, T = 8, 8, 2
     states = [B.State(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold, wl.sparsity,
                       seed=I.BASE_SEED + w) for w in range(NW)]
     L, off = states[0].arena_len, states[0].arena_offset
