@@ -3,8 +3,10 @@
 
 One *step* is one pass of the whole hot path over one batch of synthetic
 gradients: for each of the N_w simulated workers one dgc_compress (clip,
-momentum correction, exact top-k selection, emission, masking), then one
-dgc_decode_accumulate over the N_w sparse lists and one dgc_apply_sgd.
+momentum correction, exact top-k selection, emission, masking), then the
+decode of the N_w sparse lists into the dense gradient and the SGD step
+(dgc_decode_accumulate_sgd: both in one pass; --separate-receive runs
+dgc_decode_accumulate and dgc_apply_sgd as two calls).
 
 Headline metric: compressed gradient elements per second (all workers),
 inputs resident in HBM.  Beside it: the roofline of the dominant kernel
@@ -197,8 +199,16 @@ def run_ours(args):
             for i, s_ in enumerate(side):
                 ev_join[i].record(s_)
                 main_stream.wait_event(ev_join[i])
-        B.decode_accumulate(out_i, out_v, dense, ws)
-        B.apply_sgd(weights, dense, LR)
+        receive_side()
+
+    def receive_side():
+        # Alg. 4 aggregation + update lines: the dense gradient is written and the weights are
+        # updated; one pass by default, the two separate calls with --separate-receive
+        if args.separate_receive:
+            B.decode_accumulate(out_i, out_v, dense, ws)
+            B.apply_sgd(weights, dense, LR)
+        else:
+            B.decode_accumulate_sgd(out_i, out_v, dense, weights, LR, ws)
 
     def barrier():
         torch.cuda.synchronize()
@@ -235,8 +245,7 @@ def run_ours(args):
     for t in range(W + K, W + 2 * K):          # one stream: overlapped kernels cannot be timed
         for w in range(NW):
             states[w].compress(pool[w][t % POOL], out_i[w], out_v[w])
-        B.decode_accumulate(out_i, out_v, dense, ws)
-        B.apply_sgd(weights, dense, LR)
+        receive_side()
     torch.cuda.synchronize()
     stage_ms = np.concatenate([s.profile_read(K) for s in states], axis=0)
     kern_ms = stage_ms[:, 2]
@@ -271,6 +280,8 @@ def run_ours(args):
         B.apply_sgd(weights, dense, LR)
 
     receive = {"decode_plus_sgd_ms": _time(_dense_receive),
+               "one_pass_decode_sgd_ms": _time(
+                   lambda: B.decode_accumulate_sgd(out_i, out_v, dense, weights, LR, ws)),
                "fused_sparse_decode_sgd_ms": _time(
                    lambda: B.decode_apply_sgd(out_i, out_v, weights, LR, ws))}
 
@@ -297,8 +308,7 @@ def run_ours(args):
             for w in range(NW):
                 out_i[w].copy_(hi[w], non_blocking=True)
                 out_v[w].copy_(hv[w], non_blocking=True)
-            B.decode_accumulate(out_i, out_v, dense, ws)
-            B.apply_sgd(weights, dense, LR)
+            receive_side()
 
         e2e_step(0)
         barrier()
@@ -331,7 +341,10 @@ def run_ours(args):
         "config": {"workload": wl.name, "tensors": len(wl.shapes), "elements": total,
                    "simulated_workers": NW, "sparsity": wl.sparsity, "momentum": wl.momentum,
                    "clip_threshold": wl.clip_threshold, "sample_ratio": wl.sample_ratio,
-                   "nnz_per_worker": nnz, "streams": NS, "l2": "inputs larger than L2 (each worker streams "
+                   "nnz_per_worker": nnz, "streams": NS,
+                   "receive": "dgc_decode_accumulate + dgc_apply_sgd" if args.separate_receive
+                   else "dgc_decode_accumulate_sgd (dense gradient and SGD step in one pass)",
+                   "l2": "inputs larger than L2 (each worker streams "
                    f"{3 * L * 4 / 1e6:.0f} MB of g,u,v; {NW} workers cycle)",
                    "parallelism": "replicas only" if world > 1 else "1 GPU"},
         "roofline": {"bound": "hbm", "kernel": "k_update_emit", "achieved": achieved,
@@ -448,8 +461,7 @@ def run_schedule(args):
                     ev = torch.cuda.Event()
                     ev.record(q)
                     main_stream.wait_event(ev)
-            B.decode_accumulate(out_i, out_v, dense, ws)
-            B.apply_sgd(weights, dense, LR)
+            B.decode_accumulate_sgd(out_i, out_v, dense, weights, LR, ws)
 
         for _ in range(3):
             step(it)
@@ -575,6 +587,8 @@ def main():
     ap.add_argument("--clip", type=float, default=None, help="override thr_G (0 = off)")
     ap.add_argument("--sparsity", type=float, default=None)
     ap.add_argument("--streams", type=int, default=8, help="streams the workers' compress calls use")
+    ap.add_argument("--separate-receive", action="store_true",
+                    help="decode and SGD as two calls instead of the one-pass entry point")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -233,6 +233,16 @@ int32_t dgc_decode_runlength(const uint16_t* runs, const float* values, int64_t 
 int64_t dgc_runlength_max_entries(int64_t nnz, int64_t dense_len);
 int64_t dgc_runlength_workspace_bytes(int64_t entries);
 
+/* dgc_decode_accumulate and dgc_apply_sgd in one pass (Alg. 4, aggregation and update lines):
+ * writes the dense gradient to dense_out exactly as dgc_decode_accumulate does and updates
+ * w[i] <- w[i] - lr * dense_out[i] exactly as dgc_apply_sgd does, while the tile of the
+ * gradient is still on chip (12 B/element moved instead of 16).  dense_out and w: device,
+ * len floats, 16-byte aligned, distinct.  Other arguments as for dgc_decode_accumulate. */
+int32_t dgc_decode_accumulate_sgd(int32_t num_workers, const int32_t* const* idx_lists,
+                                  const float* const* val_lists, const int64_t* nnz,
+                                  float* dense_out, float* w, int64_t len, float lr,
+                                  void* workspace, int64_t workspace_bytes, void* stream);
+
 /* Synchronises `stream`, then reports counters of the last dgc_compress. */
 int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out);
 

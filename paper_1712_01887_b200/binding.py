@@ -64,6 +64,10 @@ _sigs = {
                                                       ctypes.POINTER(_vp), _i64p, _vp,
                                                       ctypes.c_int64, _vp]),
     "dgc_apply_sgd": (ctypes.c_int32, [_vp, _vp, ctypes.c_int64, ctypes.c_float, _vp]),
+    "dgc_decode_accumulate_sgd": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
+                                                   ctypes.POINTER(_vp), _i64p, _vp, _vp,
+                                                   ctypes.c_int64, ctypes.c_float, _vp,
+                                                   ctypes.c_int64, _vp]),
     "dgc_decode_apply_sgd": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
                                               ctypes.POINTER(_vp), _i64p, _vp, ctypes.c_int64,
                                               ctypes.c_float, _vp, ctypes.c_int64, _vp]),
@@ -255,6 +259,25 @@ def decode_accumulate(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[tor
                                       dense_out.numel(), workspace.data_ptr(),
                                       workspace.numel() * workspace.element_size(),
                                       _stream(stream)), "dgc_decode_accumulate")
+
+
+def decode_accumulate_sgd(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[torch.Tensor],
+                          dense_out: torch.Tensor, w: torch.Tensor, lr: float,
+                          workspace: torch.Tensor, stream=None,
+                          nnz: Optional[Sequence[int]] = None) -> None:
+    """dense_out <- sum of the workers' lists and w <- w - lr * dense_out in one pass."""
+    n = len(idx_lists)
+    ip = (_vp * n)(*[_dev(t, torch.int32) for t in idx_lists])
+    vp = (_vp * n)(*[_dev(t, torch.float32) for t in val_lists])
+    cnt = (ctypes.c_int64 * n)(*[int(c) for c in (nnz if nnz is not None
+                                                  else [t.numel() for t in idx_lists])])
+    if w.numel() != dense_out.numel():
+        raise ValueError("length mismatch")
+    _check(_lib.dgc_decode_accumulate_sgd(n, ip, vp, cnt, _dev(dense_out, torch.float32),
+                                          _dev(w, torch.float32), w.numel(), float(lr),
+                                          workspace.data_ptr(),
+                                          workspace.numel() * workspace.element_size(),
+                                          _stream(stream)), "dgc_decode_accumulate_sgd")
 
 
 def decode_apply_sgd(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[torch.Tensor],

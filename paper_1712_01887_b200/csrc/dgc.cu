@@ -627,8 +627,8 @@ int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lis
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
   launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  launch(k_decode_tiles<false>, a.num_tiles, kDecodeThreads, 0, s, a, (const int32_t*)workspace,
-                                                              dense_out, dense_len, 0.0f);
+  launch(k_decode_tiles<kDecodeDense>, a.num_tiles, kDecodeThreads, 0, s, a,
+         (const int32_t*)workspace, dense_out, (float*)nullptr, dense_len, 0.0f);
   return check_launch();
 }
 
@@ -658,8 +658,41 @@ int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_list
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
   launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  launch(k_decode_tiles<true>, a.num_tiles, kDecodeThreads, 0, s, a, (const int32_t*)workspace, w, len,
-                                                             lr);
+  launch(k_decode_tiles<kDecodeSparseSgd>, a.num_tiles, kDecodeThreads, 0, s, a,
+         (const int32_t*)workspace, w, (float*)nullptr, len, lr);
+  return check_launch();
+}
+
+int32_t dgc_decode_accumulate_sgd(int32_t num_workers, const int32_t* const* idx_lists,
+                                  const float* const* val_lists, const int64_t* nnz,
+                                  float* dense_out, float* w, int64_t len, float lr,
+                                  void* workspace, int64_t workspace_bytes, void* stream) {
+  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
+  if (!idx_lists || !val_lists || !nnz || len < 0 || len >= (int64_t)1 << 31) return DGC_EINVAL;
+  if (len == 0) return DGC_OK;
+  if (!w || !dense_out || !workspace) return DGC_EINVAL;
+  if (((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(dense_out)) & 15u) != 0)
+    return DGC_EINVAL;
+  if (workspace_bytes < dgc_decode_workspace_bytes(num_workers, len)) return DGC_ECAPACITY;
+  DecodeArgs a{};
+  int64_t max_nnz = 0;
+  for (int k = 0; k < num_workers; ++k) {
+    if (nnz[k] < 0 || nnz[k] > len) return DGC_EINVAL;
+    if (nnz[k] > 0 && (!idx_lists[k] || !val_lists[k])) return DGC_EINVAL;
+    a.idx[k] = idx_lists[k];
+    a.val[k] = val_lists[k];
+    a.nnz[k] = (int32_t)nnz[k];
+    max_nnz = std::max(max_nnz, nnz[k]);
+  }
+  a.num_workers = num_workers;
+  a.num_tiles = (int32_t)((len + kDecodeTile - 1) / kDecodeTile);
+  cudaStream_t s = as_stream(stream);
+  int32_t rc;
+  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
+  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
+  if ((rc = check_launch()) != DGC_OK) return rc;
+  launch(k_decode_tiles<kDecodeDenseSgd>, a.num_tiles, kDecodeThreads, 0, s, a,
+         (const int32_t*)workspace, dense_out, w, len, lr);
   return check_launch();
 }
 
@@ -895,6 +928,7 @@ extern "C" int32_t dgc_decode_accumulate_static(int32_t num_workers,
   const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
   launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, bounds);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  launch(k_decode_tiles<false>, a.num_tiles, kDecodeThreads, 0, s, a, bounds, dense_out, dense_len, 0.0f);
+  launch(k_decode_tiles<kDecodeDense>, a.num_tiles, kDecodeThreads, 0, s, a, bounds, dense_out,
+         (float*)nullptr, dense_len, 0.0f);
   return check_launch();
 }

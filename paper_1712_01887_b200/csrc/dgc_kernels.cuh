@@ -1445,14 +1445,20 @@ k_decode_bounds(const __grid_constant__ DecodeArgs a, int32_t* __restrict__ boun
   }
 }
 
-// SGD = false: the tile of the dense gradient is written out (zero-fill fused).
-// SGD = true (Eq. 5, third term applied directly): `dense` is the weight array; only the
-// entries some worker lists are updated, w <- w - lr * G with G summed as above -- bit for bit
-// what the dense gradient followed by k_sgd gives, because w - lr * (+0) = w.
-template <bool SGD>
+// MODE 0: the tile of the dense gradient is written out (zero-fill fused).
+// MODE 1 (Eq. 5, third term applied directly): `dense` is the weight array; only the entries
+// some worker lists are updated, w <- w - lr * G with G summed as above -- bit for bit what
+// the dense gradient followed by k_sgd gives, because w - lr * (+0) = w.
+// MODE 2: MODE 0 plus the SGD step on `weights` in the same pass (the tile of G is still in
+// shared memory when w is updated, so G is not read back): 12 B/element instead of 16.
+constexpr int kDecodeDense = 0, kDecodeSparseSgd = 1, kDecodeDenseSgd = 2;
+
+template <int MODE>
 __global__ void __launch_bounds__(kDecodeThreads)
 k_decode_tiles(const __grid_constant__ DecodeArgs a, const int32_t* __restrict__ bounds,
-               float* __restrict__ dense, long long dense_len, float lr) {
+               float* __restrict__ dense, float* __restrict__ weights, long long dense_len,
+               float lr) {
+  constexpr bool SGD = MODE == kDecodeSparseSgd;
   pdl_enter();
   __shared__ float tile[kDecodeTile];
   __shared__ uint32_t touched[kDecodeTile / 32];
@@ -1538,10 +1544,33 @@ k_decode_tiles(const __grid_constant__ DecodeArgs a, const int32_t* __restrict__
   if (rem >= kDecodeTile) {
     float4* d4 = reinterpret_cast<float4*>(dense + base);
     const float4* t4 = reinterpret_cast<const float4*>(tile);
+    if (MODE == kDecodeDenseSgd) {
+      float4* w4 = reinterpret_cast<float4*>(weights + base);
+      float4 wv[kDecodeTile / 4 / kDecodeThreads];
 #pragma unroll
-    for (int i = tid; i < kDecodeTile / 4; i += kDecodeThreads) __stcs(d4 + i, t4[i]);
+      for (int q = 0; q < kDecodeTile / 4 / kDecodeThreads; ++q)
+        wv[q] = __ldcs(w4 + q * kDecodeThreads + tid);
+#pragma unroll
+      for (int q = 0; q < kDecodeTile / 4 / kDecodeThreads; ++q) {
+        const int i = q * kDecodeThreads + tid;
+        const float4 gq = t4[i];
+        wv[q].x = __fsub_rn(wv[q].x, __fmul_rn(lr, gq.x));
+        wv[q].y = __fsub_rn(wv[q].y, __fmul_rn(lr, gq.y));
+        wv[q].z = __fsub_rn(wv[q].z, __fmul_rn(lr, gq.z));
+        wv[q].w = __fsub_rn(wv[q].w, __fmul_rn(lr, gq.w));
+        __stcs(d4 + i, gq);
+        __stcs(w4 + i, wv[q]);
+      }
+    } else {
+#pragma unroll
+      for (int i = tid; i < kDecodeTile / 4; i += kDecodeThreads) __stcs(d4 + i, t4[i]);
+    }
   } else {
-    for (int i = tid; i < (int)rem; i += kDecodeThreads) dense[base + i] = tile[i];
+    for (int i = tid; i < (int)rem; i += kDecodeThreads) {
+      dense[base + i] = tile[i];
+      if (MODE == kDecodeDenseSgd)
+        weights[base + i] = __fsub_rn(weights[base + i], __fmul_rn(lr, tile[i]));
+    }
   }
 }
 

@@ -139,4 +139,10 @@ def receive_side(idx_lists, val_lists, dense_len: int, w_init: np.ndarray, lr: f
     wf = torch.from_numpy(w_init.copy()).cuda()
     B.decode_apply_sgd(di, dv, wf, lr, ws)
     _assert_bits(wf.cpu().numpy(), wref, "weights after fused sparse decode + SGD")
+    # and the one-pass dense form: same dense gradient, same weights
+    wg = torch.from_numpy(w_init.copy()).cuda()
+    dense2 = torch.full((dense_len,), float("nan"), dtype=torch.float32, device="cuda")
+    B.decode_accumulate_sgd(di, dv, dense2, wg, lr, ws)
+    _assert_bits(dense2.cpu().numpy(), ref, "dense gradient of the one-pass decode + SGD")
+    _assert_bits(wg.cpu().numpy(), wref, "weights after the one-pass decode + SGD")
     return ref, wref
