@@ -189,6 +189,11 @@ def run_ours(args):
     ev_join = [torch.cuda.Event() for _ in range(NS)]
 
     def step(t):
+        if not args.no_batch:
+            # one call for all workers: the library overlaps their kernels itself
+            B.compress_batch(states, [pool[w][t % POOL] for w in range(NW)], out_i, out_v)
+            receive_side()
+            return
         if NS > 1:
             ev_fork.record(main_stream)
             for s_ in side:
@@ -341,7 +346,10 @@ def run_ours(args):
         "config": {"workload": wl.name, "tensors": len(wl.shapes), "elements": total,
                    "simulated_workers": NW, "sparsity": wl.sparsity, "momentum": wl.momentum,
                    "clip_threshold": wl.clip_threshold, "sample_ratio": wl.sample_ratio,
-                   "nnz_per_worker": nnz, "streams": NS,
+                   "nnz_per_worker": nnz,
+                   "compress_call": "dgc_compress per worker on %d streams" % NS if args.no_batch
+                   else "dgc_compress_batch (all workers in one call)",
+                   "streams": NS,
                    "receive": "dgc_decode_accumulate + dgc_apply_sgd" if args.separate_receive
                    else "dgc_decode_accumulate_sgd (dense gradient and SGD step in one pass)",
                    "l2": "inputs larger than L2 (each worker streams "
@@ -587,6 +595,9 @@ def main():
     ap.add_argument("--clip", type=float, default=None, help="override thr_G (0 = off)")
     ap.add_argument("--sparsity", type=float, default=None)
     ap.add_argument("--streams", type=int, default=8, help="streams the workers' compress calls use")
+    ap.add_argument("--no-batch", action="store_true",
+                    help="one dgc_compress per worker on --streams streams instead of "
+                         "dgc_compress_batch")
     ap.add_argument("--separate-receive", action="store_true",
                     help="decode and SGD as two calls instead of the one-pass entry point")
     ap.add_argument("--e2e-steps", type=int, default=5)

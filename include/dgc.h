@@ -138,6 +138,21 @@ int32_t dgc_layout(const dgc_state* st, int64_t* arena_offset, int64_t* k, int64
 int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, float* out_val,
                      int64_t capacity, void* stream);
 
+/* dgc_compress for several workers that live on one GPU (the paper's N nodes simulated in
+ * one memory): the same result as calling dgc_compress on each state in turn.  The workers'
+ * kernels are spread round robin over up to 8 internal streams, forked from and joined back
+ * into `stream`, so that one worker's short sampling, selection and emission kernels run
+ * while other workers' streaming passes keep the memory system busy; work enqueued on `stream`
+ * afterwards sees all outputs.
+ *   states[num_states]  distinct states on one device;  grad_arenas, out_idx, out_val,
+ *   capacity: host arrays [num_states] with the per-worker arguments of dgc_compress.
+ * The internal streams and events are created on the first call for a device (make that call
+ * outside stream capture) and are shared by all calls for that device: enqueue batches for one
+ * device from one host thread at a time. */
+int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
+                           const float* const* grad_arenas, int32_t* const* out_idx,
+                           float* const* out_val, const int64_t* capacity, void* stream);
+
 /* The same iteration with HOST buffers: copies grad_host (arena_len floats;
  * pinned memory makes the copy asynchronous) into a staging buffer the state
  * owns (allocated on first use), runs dgc_compress, copies the dgc_max_nnz(st)

@@ -55,6 +55,9 @@ _sigs = {
     "dgc_max_nnz": (ctypes.c_int64, [_vp]),
     "dgc_layout": (ctypes.c_int32, [_vp, _i64p, _i64p, _i64p, _i64p]),
     "dgc_compress": (ctypes.c_int32, [_vp, _vp, _vp, _vp, ctypes.c_int64, _vp]),
+    "dgc_compress_batch": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
+                                            ctypes.POINTER(_vp), ctypes.POINTER(_vp),
+                                            ctypes.POINTER(_vp), _i64p, _vp]),
     "dgc_compress_host": (ctypes.c_int32, [_vp, _vp, _vp, _vp, ctypes.c_int64, _vp]),
     "dgc_decode_accumulate": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
                                                ctypes.POINTER(_vp), _i64p, _vp, ctypes.c_int64,
@@ -241,6 +244,22 @@ class State:
         _check(_lib.dgc_state_write(self._h, None if u is None else u.ctypes.data,
                                     None if v is None else v.ctypes.data, _stream(stream)),
                "dgc_state_write")
+
+
+def compress_batch(states: Sequence["State"], grads: Sequence[torch.Tensor],
+                   out_idx: Sequence[torch.Tensor], out_val: Sequence[torch.Tensor],
+                   stream=None) -> None:
+    """dgc_compress for several workers on one GPU with overlapped kernels (same results)."""
+    n = len(states)
+    sp = (_vp * n)(*[st._h for st in states])
+    gp = (_vp * n)(*[_dev(g, torch.float32) for g in grads])
+    ip = (_vp * n)(*[_dev(t, torch.int32) for t in out_idx])
+    vp = (_vp * n)(*[_dev(t, torch.float32) for t in out_val])
+    cap = (ctypes.c_int64 * n)(*[min(a.numel(), b.numel()) for a, b in zip(out_idx, out_val)])
+    for st, g in zip(states, grads):
+        if g.numel() != st.arena_len:
+            raise ValueError("gradient arena has the wrong length")
+    _check(_lib.dgc_compress_batch(n, sp, gp, ip, vp, cap, _stream(stream)), "dgc_compress_batch")
 
 
 def decode_workspace_bytes(num_workers: int, dense_len: int) -> int:

@@ -534,3 +534,59 @@ def test_sparsity_lowered_after_creation_reallocates_scratch(P):
                 g[o:o + n] = rng.standard_normal(n).astype(np.float32)
             pair.step(g, rep, check_state=(t == 1))
     pair.close()
+
+
+def test_compress_batch_matches_oracle_per_worker(P):
+    """dgc_compress_batch (what bench.py times): all 8 workers of the ResNet-50-shaped set in
+    one call, with clipping on so that the norm kernels run ahead too; every worker bit for bit
+    against its oracle, then the one-pass receive side."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    wl = I.workload("resnet50")
+    NW, T, clip = 8, 3, 1.0
+    states = [B.State(wl.numel, NW, wl.momentum, clip, wl.sparsity, seed=I.BASE_SEED + w)
+              for w in range(NW)]
+    L, off = states[0].arena_len, states[0].arena_offset
+    oracles = [O.Worker(off, wl.numel, L, NW, wl.momentum, clip, wl.sparsity) for _ in range(NW)]
+    nnz = states[0].max_nnz
+    out_i = [torch.empty(nnz, dtype=torch.int32, device="cuda") for _ in range(NW)]
+    out_v = [torch.empty(nnz, dtype=torch.float32, device="cuda") for _ in range(NW)]
+    dense = torch.empty(L, dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.decode_workspace_bytes(NW, L), dtype=torch.uint8, device="cuda")
+    weights = torch.zeros(L, dtype=torch.float32, device="cuda")
+    w_ref = np.zeros(L, np.float32)
+    overrides = 0
+    for t in range(T):
+        hosts = []
+        for w in range(NW):
+            g = np.zeros(L, np.float32)
+            I.fill(wl, g, off, worker=w, iteration=t)
+            g *= np.float32(300.0)               # norm well above the clip threshold
+            hosts.append(g)
+        dev = [torch.from_numpy(g).cuda() for g in hosts]
+        B.compress_batch(states, dev, out_i, out_v)
+        B.decode_accumulate_sgd(out_i, out_v, dense, weights, 0.1, ws)
+        torch.cuda.synchronize()
+        res = []
+        for w in range(NW):
+            st = states[w].status()
+            snap = (oracles[w].u.copy(), oracles[w].v.copy())
+            r = oracles[w].compress(hosts[w])
+            assert abs(st.grad_norm - r.norm) <= 1e-6 * r.norm and r.coef < 1.0
+            if np.float32(st.clip_coef).tobytes() != np.float32(r.coef).tobytes():
+                oracles[w].u[:], oracles[w].v[:] = snap
+                r = oracles[w].compress(hosts[w], coef_override=st.clip_coef)
+                overrides += 1
+            assert out_i[w].cpu().numpy().tobytes() == r.idx.tobytes(), (t, w)
+            assert out_v[w].cpu().numpy().tobytes() == r.val.tobytes(), (t, w)
+            res.append(r)
+        ref = O.decode_accumulate([r.idx for r in res], [r.val for r in res], L)
+        O.apply_sgd(w_ref, ref, 0.1)
+        assert dense.cpu().numpy().tobytes() == ref.tobytes()
+        assert weights.cpu().numpy().tobytes() == w_ref.tobytes()
+    for w in range(NW):
+        u, v = states[w].read()
+        assert u.tobytes() == oracles[w].u.tobytes() and v.tobytes() == oracles[w].v.tobytes()
+    assert overrides <= 1
+    for st in states:
+        st.close()
