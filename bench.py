@@ -225,6 +225,25 @@ def run_ours(args):
     for t in range(W):
         step(t)
     barrier()
+    graphs, graph_launches = None, 0
+    if args.graph:
+        # the whole step captured once per pooled gradient and replayed: every replay is one
+        # more iteration on the same buffers (the library keeps its per-call state on the device)
+        graphs = []
+        for i in range(POOL):
+            gr = torch.cuda.CUDAGraph()
+            n0 = B.launch_count()
+            with torch.cuda.graph(gr):
+                step(i)
+            graph_launches = B.launch_count() - n0
+            graphs.append(gr)
+        eager_step = step
+
+        def step(t):                               # noqa: F811
+            graphs[t % POOL].replay()
+        for t in range(W):
+            step(t)
+        barrier()
     sampler = ClockSampler(dev)
     if rank == 0:
         sampler.start()
@@ -239,6 +258,9 @@ def run_ours(args):
     barrier()
     ms = e0.elapsed_time(e1)
     launches = B.launch_count() - launches0
+    if graphs is not None:
+        launches = graph_launches * K              # kernels inside the replayed graphs
+        del graphs
     clocks = sampler.stop() if rank == 0 else None
     ms = max_over_ranks(ms)
 
@@ -350,6 +372,7 @@ def run_ours(args):
                    "compress_call": "dgc_compress per worker on %d streams" % NS if args.no_batch
                    else "dgc_compress_batch (all workers in one call)",
                    "streams": NS,
+                   "launch": "cuda graph replay" if args.graph else "stream launches",
                    "receive": "dgc_decode_accumulate + dgc_apply_sgd" if args.separate_receive
                    else "dgc_decode_accumulate_sgd (dense gradient and SGD step in one pass)",
                    "l2": "inputs larger than L2 (each worker streams "
@@ -598,6 +621,9 @@ def main():
     ap.add_argument("--no-batch", action="store_true",
                     help="one dgc_compress per worker on --streams streams instead of "
                          "dgc_compress_batch")
+    ap.add_argument("--graph", action="store_true",
+                    help="capture the step into CUDA graphs (one per pooled gradient) and time "
+                         "their replays")
     ap.add_argument("--separate-receive", action="store_true",
                     help="decode and SGD as two calls instead of the one-pass entry point")
     ap.add_argument("--e2e-steps", type=int, default=5)

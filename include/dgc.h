@@ -134,7 +134,13 @@ int32_t dgc_layout(const dgc_state* st, int64_t* arena_offset, int64_t* k, int64
  *   capacity    >= dgc_max_nnz(st), else DGC_ECAPACITY and nothing is enqueued
  * Exactly dgc_max_nnz(st) pairs are written.  Asynchronous on `stream`; calls
  * on one state must be stream-ordered with respect to each other, and the
- * state's device must be the current device. */
+ * state's device must be the current device.
+ * Stream capture: the call only launches kernels, and what changes from call to call
+ * (the sampling seed, the bank of status counters) is derived on the device from a count
+ * of completed calls kept in device memory, so the call may be captured into a CUDA graph
+ * and replayed (with dgc_profile_enable off); each replay is one iteration on the buffers
+ * that were captured.  dgc_get_status reports the device's count.  A graph is bound to the
+ * sparsity it was captured at: capture again after dgc_set_sparsity. */
 int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, float* out_val,
                      int64_t capacity, void* stream);
 

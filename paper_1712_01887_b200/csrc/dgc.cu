@@ -423,8 +423,8 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   st->plan.sent_bits = st->d_sent_bits;
   if (cudaMemset(ptr, 0, (size_t)st->arena_len / 8) != cudaSuccess) return fail(DGC_ECUDA);
   st->plan.defer_mask = defer_mask_for(st->sparsity);
-  // scalars: partials[kMaxNormGrid] doubles, norm, diag[8] long long, coef, ticket
-  const size_t scal_bytes = (kMaxNormGrid + 1) * 8 + 8 * 8 + 16;
+  // scalars: partials[kMaxNormGrid] doubles, norm, diag[8] long long, coef, ticket, iter
+  const size_t scal_bytes = (kMaxNormGrid + 1) * 8 + 8 * 8 + 16 + 8;
   if ((rc = dev_alloc(st, &ptr, scal_bytes)) != DGC_OK) return fail(rc);
   char* sc = (char*)ptr;
   st->plan.partials = (double*)sc;
@@ -432,6 +432,7 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   st->plan.diag = (long long*)(sc + (kMaxNormGrid + 1) * 8);
   st->plan.coef = (float*)(sc + (kMaxNormGrid + 1) * 8 + 64);
   st->plan.ticket = (unsigned int*)(sc + (kMaxNormGrid + 1) * 8 + 64 + 8);
+  st->plan.iter = (long long*)(sc + (kMaxNormGrid + 1) * 8 + 64 + 16);
   if (cudaMemset(st->plan.u, 0, (size_t)st->arena_len * 4) != cudaSuccess) return fail(DGC_ECUDA);
   if (cudaMemset(st->plan.v, 0, (size_t)st->arena_len * 4) != cudaSuccess) return fail(DGC_ECUDA);
   if (cudaMemset(sc, 0, scal_bytes) != cudaSuccess) return fail(DGC_ECUDA);
@@ -501,7 +502,7 @@ static int32_t enqueue_head(dgc_state* st, const float* grad_arena, cudaStream_t
   const bool clip = st->cfg.clip_threshold > 0.0f;
   const bool nest = st->cfg.nesterov != 0;
   const float m = st->cfg.momentum;
-  const uint64_t call_seed = st->cfg.seed * 0x9E3779B97F4A7C15ull + (uint64_t)st->iterations;
+  const uint64_t call_seed = st->cfg.seed * 0x9E3779B97F4A7C15ull;   // + the device's call count
   int32_t rc;
   if (clip) {
     const double thr_local =
@@ -537,11 +538,9 @@ static int32_t enqueue_stream_pass(dgc_state* st, const float* grad_arena, cudaS
 static int32_t enqueue_tail(dgc_state* st, int32_t* out_idx, float* out_val, cudaStream_t s,
                             cudaEvent_t after_select = nullptr) {
   const Plan& p = st->plan;
-  const int parity = (int)(st->iterations & 1);
   int32_t rc;
   launch(k_select, p.num_tensors, kSelectThreads,
-         (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s, p, st->select_smem_keys,
-         parity);
+         (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s, p, st->select_smem_keys);
   if ((rc = check_launch()) != DGC_OK) return rc;
   if (p.num_big_parts > 0) {
     launch(k_big_hist<0>, p.num_big_parts, kBigThreads, 0, s, p);
@@ -550,7 +549,7 @@ static int32_t enqueue_tail(dgc_state* st, int32_t* out_idx, float* out_val, cud
     if ((rc = check_launch()) != DGC_OK) return rc;
     launch(k_big_hist<2>, p.num_big_parts, kBigThreads, 0, s, p);
     if ((rc = check_launch()) != DGC_OK) return rc;
-    launch(k_big_final, p.num_big_tensors, kSelectThreads, 0, s, p, parity);
+    launch(k_big_final, p.num_big_tensors, kSelectThreads, 0, s, p);
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (after_select) DGC_CUDA(cudaEventRecord(after_select, s));
@@ -863,6 +862,10 @@ int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out) {
   DGC_CUDA(cudaMemcpy(diag, st->plan.diag, sizeof diag, cudaMemcpyDeviceToHost));
   DGC_CUDA(cudaMemcpy(&norm, st->plan.norm, 8, cudaMemcpyDeviceToHost));
   DGC_CUDA(cudaMemcpy(&coef, st->plan.coef, 4, cudaMemcpyDeviceToHost));
+  // the device's count is the truth: a captured call replayed n times counts n times
+  long long done = 0;
+  DGC_CUDA(cudaMemcpy(&done, st->plan.iter, 8, cudaMemcpyDeviceToHost));
+  st->iterations = done;
   const int parity = (int)((st->iterations + 1) & 1);   // parity of the last call
   const bool clip = st->cfg.clip_threshold > 0.0f;
   out->grad_norm = clip ? norm : 0.0;

@@ -119,6 +119,9 @@ struct Plan {
   double* partials;
   unsigned int* ticket;
   long long* diag;           // [2][4]: flags, full_select, candidates, unused
+  long long* iter;           // compress calls completed on this state: the kernels take the
+                             // sampling seed and the counter bank from it, so that a captured
+                             // call replays correctly; k_emit_mask advances it
   float* u;
   float* v;
   // deferred masking (low sparsity): k_emit_mask records the sent entries as one bit each and
@@ -382,8 +385,9 @@ k_sumsq(Plan p, const float* __restrict__ g, double thr_local, int clip_on) {
 // reach it), keeps the few keys that reach the bound and selects among them.
 template <bool CLIP, bool NEST>
 __global__ void __launch_bounds__(kSampleThreads)
-k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t call_seed) {
+k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_base) {
   pdl_enter();
+  const uint64_t call_seed = seed_base + (uint64_t)__ldcg(p.iter);
   __shared__ uint32_t hist[kHistWords(kSampleThreads)];
   __shared__ uint32_t surv[kSampleSurvivors];
   __shared__ int sh[2];
@@ -646,8 +650,9 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
 // quota; then each part's first output slot and its share of the ties (ties go
 // to the lower index, so to the earlier part).  One block per tensor.
 __global__ void __launch_bounds__(kSelectThreads)
-k_select(Plan p, int smem_keys, int parity) {
+k_select(Plan p, int smem_keys) {
   pdl_enter();
+  const int parity = (int)(__ldcg(p.iter) & 1);
   extern __shared__ uint32_t dyn_smem[];          // [histograms | keys]
   uint32_t* hist = dyn_smem;
   uint32_t* skeys = dyn_smem + kHistWords(kSelectThreads);
@@ -1039,8 +1044,9 @@ k_big_hist(Plan p) {
 }
 
 __global__ void __launch_bounds__(kSelectThreads)
-k_big_final(Plan p, int parity) {
+k_big_final(Plan p) {
   pdl_enter();
+  const int parity = (int)(__ldcg(p.iter) & 1);
   __shared__ int sh[68];
   __shared__ int s_gt[kSelectThreads];
   __shared__ int s_eq[kSelectThreads];
@@ -1227,6 +1233,9 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   uint32_t* meq = smask + kPartSegs * kMaskStride;
   const int part = blockIdx.x;
   const int tid = threadIdx.x;
+  // the call's last kernel counts the call: nothing in this grid reads the counter, and the
+  // next call's kernels start after this grid has finished
+  if (part == 0 && tid == 0) *p.iter += 1;
   // one round of independent loads: part record, selection result, candidate count
   const PartMeta pm = load_record(p.pm + part);
   PartSel ps = load_record(p.psel + part);

@@ -590,3 +590,84 @@ def test_compress_batch_matches_oracle_per_worker(P):
     assert overrides <= 1
     for st in states:
         st.close()
+
+
+def test_cuda_graph_replay_matches_oracle(P):
+    """One whole step (dgc_compress_batch of all workers + the one-pass receive side) captured
+    into a CUDA graph and replayed: every replay is one more iteration of Algorithm 4 on the
+    captured buffers, bit for bit against the oracle.  What changes between calls (sampling
+    seed, status counter bank) must therefore come from the device, not from the host call."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    wl = I.workload("lstm_small")
+    NW, clip, lr = 3, wl.clip_threshold, 0.05
+    states = [B.State(wl.numel, NW, wl.momentum, clip, wl.sparsity, seed=I.BASE_SEED + w)
+              for w in range(NW)]
+    L, off = states[0].arena_len, states[0].arena_offset
+    oracles = [O.Worker(off, wl.numel, L, NW, wl.momentum, clip, wl.sparsity) for _ in range(NW)]
+    nnz = states[0].max_nnz
+    g_dev = [torch.zeros(L, dtype=torch.float32, device="cuda") for _ in range(NW)]
+    out_i = [torch.empty(nnz, dtype=torch.int32, device="cuda") for _ in range(NW)]
+    out_v = [torch.empty(nnz, dtype=torch.float32, device="cuda") for _ in range(NW)]
+    dense = torch.empty(L, dtype=torch.float32, device="cuda")
+    ws = torch.empty(B.decode_workspace_bytes(NW, L), dtype=torch.uint8, device="cuda")
+    weights = torch.zeros(L, dtype=torch.float32, device="cuda")
+    w_ref = np.zeros(L, np.float32)
+
+    overrides = []
+
+    def step():
+        B.compress_batch(states, g_dev, out_i, out_v)
+        B.decode_accumulate_sgd(out_i, out_v, dense, weights, lr, ws)
+
+    def load(t):
+        hosts = []
+        for w in range(NW):
+            g = np.zeros(L, np.float32)
+            I.fill(wl, g, off, worker=w, iteration=t)
+            g *= np.float32(40.0)                # clipping active
+            g_dev[w].copy_(torch.from_numpy(g))
+            hosts.append(g)
+        return hosts
+
+    def check(hosts, t):
+        torch.cuda.synchronize()
+        res = []
+        for w in range(NW):
+            st = states[w].status()
+            assert st.iterations == t + 1
+            snap = (oracles[w].u.copy(), oracles[w].v.copy())
+            r = oracles[w].compress(hosts[w])
+            assert abs(st.grad_norm - r.norm) <= 1e-6 * r.norm and r.coef < 1.0
+            if np.float32(st.clip_coef).tobytes() != np.float32(r.coef).tobytes():
+                oracles[w].u[:], oracles[w].v[:] = snap
+                r = oracles[w].compress(hosts[w], coef_override=st.clip_coef)
+                overrides.append((t, w))
+            assert out_i[w].cpu().numpy().tobytes() == r.idx.tobytes(), (t, w)
+            assert out_v[w].cpu().numpy().tobytes() == r.val.tobytes(), (t, w)
+            res.append(r)
+        ref = O.decode_accumulate([r.idx for r in res], [r.val for r in res], L)
+        O.apply_sgd(w_ref, ref, lr)
+        assert dense.cpu().numpy().tobytes() == ref.tobytes(), t
+        assert weights.cpu().numpy().tobytes() == w_ref.tobytes(), t
+
+    hosts = load(0)
+    step()                                       # plain call first (creates the side streams)
+    check(hosts, 0)
+    graph = torch.cuda.CUDAGraph()
+    hosts = load(1)
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph):
+        step()                                   # captured, not run
+    for t in range(1, 5):
+        if t > 1:
+            hosts = load(t)
+        graph.replay()
+        check(hosts, t)
+    for w in range(NW):
+        u, v = states[w].read()
+        assert u.tobytes() == oracles[w].u.tobytes() and v.tobytes() == oracles[w].v.tobytes()
+    assert len(overrides) <= 1
+    del graph
+    for st in states:
+        st.close()
