@@ -290,6 +290,13 @@ int32_t dgc_get_thresholds(dgc_state* st, void* stream, uint32_t* kth_key, int32
 int32_t dgc_state_read(dgc_state* st, float* u_host, float* v_host, void* stream);
 int32_t dgc_state_write(dgc_state* st, const float* u_host, const float* v_host, void* stream);
 
+/* Checkpoint / resume, the third piece of a worker's state: sets the count of completed
+ * dgc_compress calls (dgc_status.iterations of the checkpointed state).  The exact top-k
+ * result does not depend on it; the sample positions do, so the paper-literal mode
+ * (select_mode 1) resumes bit-identically only with the count restored.  Synchronous on
+ * `stream`; clears the status counters of the last call.  iterations >= 0, else DGC_EINVAL. */
+int32_t dgc_state_set_iterations(dgc_state* st, int64_t iterations, void* stream);
+
 /* Measurement aid (not part of the method): after dgc_profile_enable(st, n) the
  * next n dgc_compress calls record CUDA events on the call's stream at their
  * stage boundaries.  dgc_profile_read waits for the recorded calls and returns,

@@ -85,6 +85,7 @@ _sigs = {
     "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_write": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
+    "dgc_state_set_iterations": (ctypes.c_int32, [_vp, ctypes.c_int64, _vp]),
     "dgc_profile_enable": (ctypes.c_int32, [_vp, ctypes.c_int32]),
     "dgc_profile_read": (ctypes.c_int32, [_vp, _vp, ctypes.c_int32,
                                           ctypes.POINTER(ctypes.c_int32)]),
@@ -244,6 +245,10 @@ class State:
         _check(_lib.dgc_state_write(self._h, None if u is None else u.ctypes.data,
                                     None if v is None else v.ctypes.data, _stream(stream)),
                "dgc_state_write")
+
+    def set_iterations(self, iterations: int, stream=None) -> None:
+        _check(_lib.dgc_state_set_iterations(self._h, int(iterations), _stream(stream)),
+               "dgc_state_set_iterations")
 
 
 def compress_batch(states: Sequence["State"], grads: Sequence[torch.Tensor],

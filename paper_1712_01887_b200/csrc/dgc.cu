@@ -959,6 +959,19 @@ int32_t dgc_state_write(dgc_state* st, const float* u_host, const float* v_host,
   return DGC_OK;
 }
 
+int32_t dgc_state_set_iterations(dgc_state* st, int64_t iterations, void* stream) {
+  if (!st || !st->alive) return DGC_ESTATE;
+  if (iterations < 0) return DGC_EINVAL;
+  cudaStream_t s = as_stream(stream);
+  DGC_CUDA(cudaStreamSynchronize(s));
+  const long long zeros[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  const long long it = iterations;
+  DGC_CUDA(cudaMemcpy(st->plan.diag, zeros, sizeof zeros, cudaMemcpyHostToDevice));
+  DGC_CUDA(cudaMemcpy(st->plan.iter, &it, 8, cudaMemcpyHostToDevice));
+  st->iterations = iterations;
+  return DGC_OK;
+}
+
 }  // extern "C"
 
 // ====================================================================== allocation-free decode

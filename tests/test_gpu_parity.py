@@ -671,3 +671,55 @@ def test_cuda_graph_replay_matches_oracle(P):
     del graph
     for st in states:
         st.close()
+
+
+def test_checkpoint_resume_paper_literal_needs_the_call_count(P):
+    """Paper-literal mode draws its sample from (seed, call count): a resumed state gives the
+    uninterrupted run's lists only with u, v AND the count restored (dgc_state_set_iterations);
+    the resumed calls are also checked against the oracle at the restored iteration numbers."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    numel, seed, s = [300000, 9000, 70001], 31, 0.999
+    a = B.State(numel, 2, 0.9, 0.0, s, seed=seed, select_mode=1)
+    L, off = a.arena_len, a.arena_offset
+    cpu = O.Worker(off, numel, L, 2, 0.9, 0.0, s)
+    rng = np.random.default_rng(12)
+    gs = []
+    for _ in range(5):
+        g = np.zeros(L, np.float32)
+        for o, n in zip(off, numel):
+            g[o:o + n] = rng.standard_normal(n).astype(np.float32)
+        gs.append(g)
+    oi = torch.empty(a.max_nnz, dtype=torch.int32, device="cuda")
+    ov = torch.empty(a.max_nnz, dtype=torch.float32, device="cuda")
+    for t in range(3):
+        a.compress(torch.from_numpy(gs[t]).cuda(), oi, ov)
+        O.compress_sampled(cpu, gs[t], seed=seed, iteration=t)
+    u, v = a.read()
+    done = a.status().iterations
+    assert done == 3
+    b = B.State(numel, 2, 0.9, 0.0, s, seed=seed, select_mode=1)
+    b.write(u, v)
+    b.set_iterations(done)
+    assert b.status().iterations == 3
+    oi2, ov2 = torch.empty_like(oi), torch.empty_like(ov)
+    for t in range(3, 5):
+        gd = torch.from_numpy(gs[t]).cuda()
+        a.compress(gd, oi, ov)
+        b.compress(gd, oi2, ov2)
+        na, pa = a.nnz()
+        nb, pb = b.nnz()
+        r, nnz = O.compress_sampled(cpu, gs[t], seed=seed, iteration=t)
+        assert na == nb == r.idx.size and pa.tolist() == pb.tolist() == nnz.tolist()
+        assert oi2[:nb].cpu().numpy().tobytes() == r.idx.tobytes()
+        assert ov2[:nb].cpu().numpy().tobytes() == r.val.tobytes()
+        assert torch.equal(oi[:na], oi2[:nb])
+        assert torch.equal(ov[:na].view(torch.int32), ov2[:nb].view(torch.int32))
+    ua, va = a.read()
+    ub, vb = b.read()
+    assert ua.tobytes() == ub.tobytes() == cpu.u.tobytes()
+    assert va.tobytes() == vb.tobytes() == cpu.v.tobytes()
+    with pytest.raises(Exception):
+        b.set_iterations(-1)
+    a.close()
+    b.close()
