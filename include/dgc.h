@@ -49,6 +49,10 @@ extern "C" {
 #define DGC_FLAG_FULL_SELECT      2  /* a tensor needed the full-tensor selection   */
 #define DGC_FLAG_CAND_OVERFLOW    4  /* sampled threshold let too many entries pass */
 #define DGC_FLAG_CAND_SHORT       8  /* sampled threshold let fewer than k pass     */
+#define DGC_FLAG_TIE_FILL        16  /* fewer than k entries of a tensor exceeded   */
+                                     /* the sample's key: entries tied with it (all */
+                                     /* zeros, few distinct magnitudes) complete    */
+                                     /* the list, lowest indices first; not slow    */
 
 typedef struct dgc_state dgc_state;   /* opaque */
 
@@ -126,8 +130,11 @@ int32_t dgc_layout(const dgc_state* st, int64_t* arena_offset, int64_t* k, int64
  *   out: their (arena index, v) pairs, ascending index, at out_offset[j]
  *   v <- 0, u <- 0 at those entries (momentum factor masking)
  * A seeded sample of |v| only proposes a threshold; the result is always the
- * exact top-k_j set (if the proposal lets fewer than k_j or too many entries
- * pass, that tensor is selected from the whole of v instead, see dgc_status).
+ * exact top-k_j set.  Tensors with masses of equal magnitudes (all zeros, sign
+ * gradients) are completed from the tied entries of lowest index without a
+ * selection (DGC_FLAG_TIE_FILL); if the proposal otherwise lets fewer than k_j or
+ * too many entries pass, that tensor is selected from the whole of v instead
+ * (slow, see dgc_status).
  *   grad_arena  device, const, arena_len floats, 16-byte aligned; not modified
  *   out_idx     device, capacity int32   (index into the arena)
  *   out_val     device, capacity floats

@@ -26,6 +26,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 OK, EINVAL, ENOMEM, ECAPACITY, ECUDA, ESTATE = 0, -1, -2, -3, -4, -5
 FLAG_NONFINITE_NORM, FLAG_FULL_SELECT, FLAG_CAND_OVERFLOW, FLAG_CAND_SHORT = 1, 2, 4, 8
+FLAG_TIE_FILL = 16
 ARENA_ALIGN = 512
 MAX_DECODE_WORKERS = 64
 

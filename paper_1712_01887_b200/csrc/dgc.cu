@@ -246,6 +246,8 @@ int32_t upload_plan(dgc_state* st, bool first) {
   const size_t o_psel = o; o = up16(o + P * sizeof(PartSel));
   const size_t o_pcount = o; o = up16(o + P * 4);
   const size_t o_pthr = o; o = up16(o + P * 4);
+  const size_t o_peq = o; o = up16(o + P * 4);
+  const size_t o_ptie = o; o = up16(o + P * 4);
   const size_t o_kth = o; o = up16(o + T * 4);
   const size_t o_cand = o; o = up16(o + T * 4);
   const size_t o_nnz = o; o = up16(o + T * 4);
@@ -284,6 +286,8 @@ int32_t upload_plan(dgc_state* st, bool first) {
   p.psel = (PartSel*)(d + o_psel);
   p.p_count = (int32_t*)(d + o_pcount);
   p.p_thr = (uint32_t*)(d + o_pthr);
+  p.p_eq = (int32_t*)(d + o_peq);
+  p.p_tie = (uint32_t*)(d + o_ptie);
   p.t_kth = (uint32_t*)(d + o_kth);
   p.t_cand = (int32_t*)(d + o_cand);
   p.t_nnz = (int32_t*)(d + o_nnz);
@@ -870,7 +874,7 @@ int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out) {
   const bool clip = st->cfg.clip_threshold > 0.0f;
   out->grad_norm = clip ? norm : 0.0;
   out->clip_coef = clip ? coef : 1.0f;
-  out->flags = (int32_t)(diag[parity * 4 + 0] & 0xF);
+  out->flags = (int32_t)(diag[parity * 4 + 0] & 0x1F);
   if (clip && !std::isfinite(norm)) out->flags |= DGC_FLAG_NONFINITE_NORM;
   out->iterations = st->iterations;
   out->full_select_last = diag[parity * 4 + 1];

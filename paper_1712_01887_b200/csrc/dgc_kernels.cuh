@@ -95,6 +95,12 @@ struct Plan {
   PartSel* psel;
   int32_t* p_count;          // candidates appended per part (reset by k_emit_mask)
   uint32_t* p_thr;           // proposed threshold per part (0 for tensors that are not sampled)
+  uint32_t* p_tie;           // per part, written with p_thr: 1 if the sample held its rank-th
+                             // key more than once (masses of equal magnitudes are possible):
+                             // only then does k_update_emit count the part's tied entries
+  int32_t* p_eq;             // entries per part whose key is p_thr - 1, the sample's rank-th key
+                             // (counted by k_update_emit, reset by k_emit_mask): what completes
+                             // the list when fewer than k entries exceed that key
   int32_t* t_nnz;            // per tensor: entries sent by the last call (paper-literal mode)
   int32_t literal;           // 1: paper-literal sampled selection (Sec. 5), variable count
   uint32_t* t_kth;           // per tensor: threshold of the last call (reporting)
@@ -222,7 +228,7 @@ __device__ __forceinline__ void block_excl_scan2(int a, int b, int* sh, int& ea,
 // of warps, so that the integer atomics of different warps do not collide;
 // they are folded into one of two alternating 256-bin histograms, in which
 // warp 0 finds the digit.  hist: kHistWords(blockDim.x) words of shared
-// memory, sh: 2 words.  blockDim.x is a multiple of 256, at least 512.
+// memory, sh: 3 words.  blockDim.x is a multiple of 256, at least 512.
 // Returns the key; n_gt = number of keys strictly greater.
 __host__ __device__ constexpr int kHistCopies(int threads) { return threads / 32 < 16 ? threads / 32 : 16; }
 __host__ __device__ constexpr int kHistWords(int threads) { return kHistCopies(threads) * 257 + 512; }
@@ -232,7 +238,7 @@ __host__ __device__ constexpr int kHistWords(int threads) { return kHistCopies(t
 template <int THREADS, bool PRIVATE = true, class ForEach>
 __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank, uint32_t base,
                                                       uint32_t maxkey, uint32_t* hist, int* sh,
-                                                      int& n_gt) {
+                                                      int& n_gt, int* n_eq = nullptr) {
   // THREADS = blockDim.x, a compile-time constant so that the slicing below costs no divisions
   constexpr int nt = THREADS;
   const int tid = threadIdx.x, lane = tid & 31;
@@ -283,7 +289,12 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
         uint32_t c = excl;
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          if (c + loc[q] >= (uint32_t)remaining) { sh[0] = hi - q; sh[1] = (int)c; break; }
+          if (c + loc[q] >= (uint32_t)remaining) {
+            sh[0] = hi - q;
+            sh[1] = (int)c;
+            sh[2] = (int)loc[q];     // after the last pass: keys equal to the result
+            break;
+          }
           c += loc[q];
         }
       }
@@ -296,6 +307,8 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
     remaining -= sh[1];
   }
   n_gt = rank - remaining;
+  // keys equal to the result: the chosen bin of the last pass (no pass: every key is maxkey)
+  if (n_eq) *n_eq = passes == 0 ? 0x7FFFFFFF : sh[2];
   return base + prefix;
 }
 
@@ -390,7 +403,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   const uint64_t call_seed = seed_base + (uint64_t)__ldcg(p.iter);
   __shared__ uint32_t hist[kHistWords(kSampleThreads)];
   __shared__ uint32_t surv[kSampleSurvivors];
-  __shared__ int sh[2];
+  __shared__ int sh[3];
   __shared__ int s_cnt;
   __shared__ uint32_t s_max;
   __shared__ int s_last;
@@ -460,7 +473,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   __syncthreads();
   const uint32_t kmax = s_max;
   const int owners = min(G, kSampleThreads);          // threads that hold at least one group
-  int n_gt;
+  int n_gt, n_eq = 0;
   uint32_t kth = 0;
   bool done = false;
   if (rank <= owners) {
@@ -500,7 +513,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
               f(i < ns, i < ns ? surv[i] : low);
             }
           },
-          rank, low, kmax, hist, sh, n_gt);
+          rank, low, kmax, hist, sh, n_gt, &n_eq);
       done = true;
     }
   }
@@ -517,12 +530,18 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
             f(i < G, kk.w);
           }
         },
-        rank, 0u, kmax, hist, sh, n_gt);
+        rank, 0u, kmax, hist, sh, n_gt, &n_eq);
   }
-  // exact mode: a proposal of 0 would let every entry through, so insist on non-zero
-  // magnitude.  Paper-literal mode: the mask is "|v| > thr" with thr the sample's rank-k_s key.
-  const uint32_t thr = p.literal ? kth + 1u : (kth > 1u ? kth : 1u);
-  for (int q = tid; q < t.part_num; q += kSampleThreads) p.p_thr[t.part_first + q] = thr;
+  // candidates are the entries that EXCEED the sample's rank-th key (p_thr = key + 1): entries
+  // tied with it are only counted (p_eq), so that a tensor with masses of equal magnitudes (all
+  // zeros, a few distinct values) neither floods the candidate lists nor needs a selection.
+  // Paper-literal mode has the same mask: "|v| > thr", thr the sample's rank-k_s key.
+  const uint32_t thr = kth + 1u;
+  const uint32_t tie_on = n_eq > 1 ? 1u : 0u;     // the sample repeats its rank-th key
+  for (int q = tid; q < t.part_num; q += kSampleThreads) {
+    p.p_thr[t.part_first + q] = thr;
+    p.p_tie[t.part_first + q] = tie_on;
+  }
 }
 
 // ------------------------------------------------------------------ K3: fused momentum correction + candidate emission
@@ -555,6 +574,7 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
     const int part = __ldg(p.seg_part + seg);
     const PartMeta pm = load_record(p.pm + part);
     const uint32_t thr = __ldcg(p.p_thr + part);
+    const bool tie_on = __ldcg(p.p_tie + part) != 0u;
     const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
     const int end = pm.end;
     const bool full = base + kSeg <= end;
@@ -584,6 +604,17 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
       flags |= (uint32_t)(mag_key(vv[i].z) >= thr) << (4 * i + 2);
       flags |= (uint32_t)(mag_key(vv[i].w) >= thr) << (4 * i + 3);
     }
+    uint32_t ties = 0;    // same layout: the element's key is thr - 1, the sample's rank-th key
+    if (tie_on) {         // warp-uniform; off unless the sample showed repeated magnitudes
+      const uint32_t tie_key = thr - 1u;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        ties |= (uint32_t)(mag_key(vv[i].x) == tie_key) << (4 * i + 0);
+        ties |= (uint32_t)(mag_key(vv[i].y) == tie_key) << (4 * i + 1);
+        ties |= (uint32_t)(mag_key(vv[i].z) == tie_key) << (4 * i + 2);
+        ties |= (uint32_t)(mag_key(vv[i].w) == tie_key) << (4 * i + 3);
+      }
+    }
     if (full) {
 #pragma unroll
       for (int i = 0; i < 4; ++i) __stcs(u4 + q0 + i * 32, uu[i]);
@@ -607,6 +638,11 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
         }
       }
       flags &= valid;
+      ties &= valid;
+    }
+    if (tie_on && __any_sync(0xFFFFFFFFu, ties != 0)) {
+      const int c = __reduce_add_sync(0xFFFFFFFFu, __popc(ties));
+      if (lane == 0) atomicAdd(p.p_eq + part, c);
     }
     if (__any_sync(0xFFFFFFFFu, flags != 0)) {
       // per-lane counts of the four float4 rows packed one per byte (row totals <= 128)
@@ -649,6 +685,51 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
 // the tensor's candidates, the number of strictly larger ones and the tie
 // quota; then each part's first output slot and its share of the ties (ties go
 // to the lower index, so to the earlier part).  One block per tensor.
+// Tie-fill selection.  The candidates are the entries that exceed the sample's rank-th key
+// (p_thr - 1).  If fewer than k exist but the entries tied with that key make up the rest, the
+// exact top-k needs no selection: all candidates, then the k - total tied entries of lowest
+// index; the threshold is that key.  Per part, its candidates are "greater" and its p_eq
+// entries are ties; k_emit_mask finds the tied entries by reading the part (PartSel.dense == 2).
+// This is the path of a tensor that is all or almost all zeros (a frozen layer, unused
+// embedding rows: the key is 0) or holds a few distinct magnitudes (sign or low-bit
+// gradients).  Returns false, having written nothing, if the ties do not suffice.
+__device__ __forceinline__ bool tie_fill_parts(const Plan& p, int p0, int pn, int k, int total,
+                                               int out_off, uint32_t kth, int* sh) {
+  const int tid = threadIdx.x;
+  int mine = 0;
+  for (int q = tid; q < pn; q += kSelectThreads) mine += __ldcg(p.p_eq + p0 + q);
+  int e1, e2, eq_total, t2;
+  block_excl_scan2(mine, 0, sh, e1, e2, eq_total, t2);
+  __syncthreads();
+  if (total + eq_total < k) return false;
+  const int quota = k - total;
+  int run_gt = 0, run_eq = 0;
+  for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+    const int q = q0 + tid;
+    int gt = 0, eq = 0;
+    if (q < pn) {
+      gt = __ldcg(p.p_count + p0 + q);
+      eq = __ldcg(p.p_eq + p0 + q);
+    }
+    int bg, be, tg, te;
+    block_excl_scan2(gt, eq, sh, bg, be, tg, te);
+    bg += run_gt;
+    be += run_eq;
+    if (q < pn) {
+      PartSel ps;
+      ps.kth = kth;
+      ps.quota = max(0, min(quota - be, eq));
+      ps.out_base = out_off + bg + min(be, quota);
+      ps.dense = 2;
+      p.psel[p0 + q] = ps;
+    }
+    run_gt += tg;
+    run_eq += te;
+    __syncthreads();
+  }
+  return true;
+}
+
 __global__ void __launch_bounds__(kSelectThreads)
 k_select(Plan p, int smem_keys) {
   pdl_enter();
@@ -717,6 +798,19 @@ k_select(Plan p, int smem_keys) {
   const bool lit_own = literal && t.groups == 0;
   const bool lit_own_all = lit_own && k + 1 > total;
   const int rank = lit_own ? k + 1 : k;
+  if (!overflow && !literal && total < k && t.groups > 0) {
+    const uint32_t tie_key = __ldcg(p.p_thr + p0) - 1u;
+    if (tie_fill_parts(p, p0, pn, k, total, t.out_off, tie_key, sh)) {
+      if (tid == 0) {
+        p.t_kth[j] = tie_key;
+        p.t_cand[j] = total;
+        p.t_nnz[j] = k;
+        atomicOr((unsigned long long*)&p.diag[parity * 4 + 0], (unsigned long long)DGC_FLAG_TIE_FILL);
+        atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
+      }
+      return;
+    }
+  }
   if (overflow || (!literal && total < k)) {
     if (tid == 0) p.t_nnz[j] = k;
     // full-selection path: k_emit_mask's block of the tensor's first part does it
@@ -1068,13 +1162,20 @@ k_big_final(Plan p) {
   block_excl_scan2(mine, over, sh, ex, exo, total, overflow);
   __syncthreads();
   const bool literal = p.literal != 0;
-  const bool dense = overflow != 0 || (!literal && total < k);
+  uint32_t kth = 0;
+  bool tie_fill = false;
+  if (overflow == 0 && !literal && total < k) {
+    kth = __ldcg(p.p_thr + p0) - 1u;
+    tie_fill = tie_fill_parts(p, p0, pn, k, total, t.out_off, kth, sh);
+  }
+  const bool dense = !tie_fill && (overflow != 0 || (!literal && total < k));
   // paper-literal mode: at most 2k passed the sampled threshold -> all of them are sent
   const bool all_pass = literal && !dense && total <= 2 * k;
   const int out_off = literal ? 0 : t.out_off;
-  uint32_t kth = 0;
   int quota = 0;
-  if (all_pass) {
+  if (tie_fill) {
+    // PartSel records already written
+  } else if (all_pass) {
     kth = __ldcg(p.p_thr + p0) - 1u;            // every candidate exceeds it
     int run = 0;
     for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
@@ -1148,6 +1249,8 @@ k_big_final(Plan p) {
       p.t_kth[j] = kth;
       p.t_cand[j] = total;
       atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
+      if (tie_fill)
+        atomicOr((unsigned long long*)&p.diag[parity * 4 + 0], (unsigned long long)DGC_FLAG_TIE_FILL);
     }
     p.t_nnz[j] = all_pass ? total : k;
   }
@@ -1255,9 +1358,9 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
     tensor_first = s_first;
     ps.out_base += tensor_first;
   }
-  if (ps.dense) {
+  if (ps.dense == 1) {
     __syncthreads();
-    if (tid == 0) p.p_count[part] = 0;
+    if (tid == 0) { p.p_count[part] = 0; p.p_eq[part] = 0; }
     if (p.defer_mask && tid < pm.nseg) {
       // the full-selection path zeroes u and v itself: nothing is pending for this part
       uint4* dst = reinterpret_cast<uint4*>(p.sent_bits + (size_t)(pm.seg0 + tid) * 16);
@@ -1284,7 +1387,7 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   }
   for (int i = tid; i < 2 * kPartSegs * kMaskStride; i += kEmitThreads) smask[i] = 0u;
   __syncthreads();
-  if (tid == 0) p.p_count[part] = 0;          // ready for the next call
+  if (tid == 0) { p.p_count[part] = 0; p.p_eq[part] = 0; }   // ready for the next call
   // mark the candidates that reach the threshold: one bit per element of the part
   int locs[kEmitRegs];
 #pragma unroll
@@ -1321,6 +1424,31 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
     }
   }
   __syncthreads();
+  const bool tie_fill = ps.dense == 2 && quota > 0;   // no quota: the part sends candidates only
+  if (tie_fill) {
+    // tie-fill selection: the ties are the part's entries whose key is the threshold; they are
+    // in no candidate list, so the part is read (one warp per segment, one ballot per word)
+    const int lane = tid & 31;
+    for (int sgm = tid >> 5; sgm < pm.nseg; sgm += kEmitThreads / 32) {
+      const int base = (pm.seg0 + sgm) * kSeg;
+#pragma unroll 1
+      for (int w0 = 0; w0 < 16; w0 += 4) {
+        float x[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const int e = base + (w0 + w) * 32 + lane;
+          x[w] = e < pm.end ? __ldcg(p.v + e) : 0.0f;
+        }
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const int e = base + (w0 + w) * 32 + lane;
+          const uint32_t word = __ballot_sync(0xFFFFFFFFu, e < pm.end && mag_key(x[w]) == kth);
+          if (lane == 0) meq[sgm * kMaskStride + w0 + w] = word;
+        }
+      }
+    }
+    __syncthreads();
+  }
   // thread s owns segment s: popcounts, then winners before each segment
   {
     int gt = 0, eq = 0;
@@ -1379,6 +1507,45 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
       const int i = i0 + b * kEmitThreads + tid;
       const uint32_t key = mag_key(v4[b]);
       if (i < count && key >= kth) emit(x4[b] - pm.seg0 * kSeg, v4[b], key);
+    }
+  }
+  if (tie_fill) {
+    // the tied entries each segment sends (lowest indices first, up to the part's quota): one
+    // warp per segment, one lane per entry of a 32-entry word
+    const int lane = tid & 31;
+    const uint32_t below = (1u << lane) - 1u;
+    for (int sgm = tid >> 5; sgm < pm.nseg; sgm += kEmitThreads / 32) {
+      int eq_before = s_eqb[sgm];
+      if (eq_before >= quota) break;             // s_eqb does not decrease with the segment
+      const int base = (pm.seg0 + sgm) * kSeg;
+      int lg = s_gtb[sgm];
+#pragma unroll 1
+      for (int w0 = 0; w0 < 16 && eq_before < quota; w0 += 4) {
+        uint32_t ew[4];
+        float x[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          ew[w] = meq[sgm * kMaskStride + w0 + w];
+          x[w] = (ew[w] >> lane) & 1u ? __ldcg(p.v + base + (w0 + w) * 32 + lane) : 0.0f;
+        }
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+          const uint32_t gw = mgt[sgm * kMaskStride + w0 + w];
+          const int eb = eq_before + __popc(ew[w] & below);
+          if (((ew[w] >> lane) & 1u) && eb < quota) {
+            const int idx = base + (w0 + w) * 32 + lane;
+            const int pos = ps.out_base + lg + __popc(gw & below) + eb;
+            out_idx[pos] = idx;
+            out_val[pos] = x[w];
+            if (!p.defer_mask) {
+              p.u[idx] = 0.0f;
+              p.v[idx] = 0.0f;
+            }
+          }
+          eq_before += __popc(ew[w]);
+          lg += __popc(gw);
+        }
+      }
     }
   }
   if (p.defer_mask && tid < pm.nseg) {

@@ -144,7 +144,7 @@ def test_heavy_ties_and_zeros(P):
     pair.close()
 
 
-def test_all_zero_gradient_takes_full_selection_and_picks_lowest_indices(P):
+def test_all_zero_gradient_is_zero_filled_with_lowest_indices(P):
     numel = [20000, 100]
     pair = P.Pair(numel, 1, 0.9, 0.0, 0.999, seed=1)
     rep = P.ParityReport()
@@ -153,7 +153,75 @@ def test_all_zero_gradient_takes_full_selection_and_picks_lowest_indices(P):
     gi, gv, st = pair.step(g, rep)
     assert gi.tolist() == list(range(20)) + [int(off[1])]
     assert not gv.any()
-    assert st.flags & 2 and st.full_select_last >= 1
+    # no selection at all: the sampled tensor's list is completed with zeros (flag 16), the
+    # small one is its own sample; nothing takes the slow full-selection path
+    assert st.flags & 16 and not st.flags & 2 and st.full_select_last == 0
+    pair.close()
+
+
+@pytest.mark.parametrize("sparsity", [0.999, 0.99])
+def test_fewer_nonzeros_than_k_zero_fill_matches_oracle(P, sparsity):
+    """Tensors with fewer non-zero entries than k (an almost unused embedding, a frozen layer):
+    all non-zeros plus the lowest-index zeros, over several iterations with momentum so that u
+    is non-zero where v was sent.  Covers one-part, multi-part and (at 99 %) multi-block-selected
+    tensors, a ragged last segment, immediate (99.9 %) and deferred (99 %) masking, and zeros
+    of either sign."""
+    numel = [700001, 1 << 22, 40000, 300, 1 << 19]
+    pair = P.Pair(numel, 1, 0.9, 0.0, sparsity, seed=4)
+    rep = P.ParityReport()
+    rng = np.random.default_rng(21)
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    # start from negative zeros in part of the state: they must be sent as they are
+    u0 = np.zeros(L, np.float32)
+    v0 = np.zeros(L, np.float32)
+    v0[off[0]:off[0] + 1000] = np.float32(-0.0)
+    u0[off[0]:off[0] + 1000] = np.float32(-0.0)
+    pair.gpu.write(u0, v0)
+    pair.cpu.u[:], pair.cpu.v[:] = u0, v0
+    nonzeros = [0, 37, 5, 0, 300]            # per tensor and iteration: all below k
+    for t in range(4):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for j, (o, n) in enumerate(zip(off, numel)):
+            if j == 0 and t < 2:
+                g[o:o + 1000] = np.float32(-0.0)
+            pos = rng.choice(n, size=nonzeros[j], replace=False)
+            g[o + pos] = rng.standard_normal(nonzeros[j]).astype(np.float32)
+        if t == 3:
+            g[off[2]:off[2] + numel[2]] = rng.standard_normal(numel[2]).astype(np.float32)
+        gi, gv, st = pair.step(g, rep)
+        assert st.flags & 16 and st.full_select_last == 0, (t, st.flags, st.full_select_last)
+        if t == 0:
+            # tensor 0: nothing non-zero, so its k lowest indices, the first 1000 of them -0.0
+            k0 = int(pair.gpu.k[0])
+            assert gi[:k0].tolist() == list(range(int(off[0]), int(off[0]) + k0))
+            assert (gv[:min(k0, 1000)].view(np.uint32) == 0x80000000).all()
+    pair.close()
+
+
+@pytest.mark.parametrize("sparsity", [0.999, 0.99])
+def test_few_distinct_magnitudes_tie_fill_matches_oracle(P, sparsity):
+    """Sign-like gradients: every entry of a tensor has one of a handful of magnitudes, so the
+    k-th largest |v| is shared by far more than k entries.  Those ties are counted, not listed
+    as candidates, and the lowest indices complete the list; no tensor may take the slow
+    full-selection path."""
+    numel = [700001, 1 << 22, 40000, 5000]
+    pair = P.Pair(numel, 1, 0.5, 0.0, sparsity, seed=9)
+    rep = P.ParityReport()
+    rng = np.random.default_rng(33)
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    for t in range(4):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for j, (o, n) in enumerate(zip(off, numel)):
+            sign = rng.integers(0, 2, size=n).astype(np.float32) * 2 - 1
+            if j == 1:
+                sign *= rng.integers(0, 3, size=n).astype(np.float32)     # magnitudes 0, 1, 2
+            g[o:o + n] = sign * np.float32(0.25)
+        gi, gv, st = pair.step(g, rep)
+        assert st.full_select_last == 0 and not st.flags & 2, (t, st.flags)
+        if t == 0:
+            assert st.flags & 16
+            k0 = int(pair.gpu.k[0])
+            assert gi[:k0].tolist() == list(range(int(off[0]), int(off[0]) + k0))
     pair.close()
 
 
