@@ -1274,14 +1274,22 @@ __device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int
   const int n = t.end - off;
   const int k = t.k;
   const float* v = p.v + off;
-  const int iters = (n + nt - 1) / nt;
   int n_gt;
   const uint32_t kth = block_select_desc<kEmitThreads>(
       [&](auto f) {
-        for (int it = 0; it < iters; ++it) {
-          const int i = it * nt + tid;
-          const bool valid = i < n;
-          f(valid, valid ? mag_key(__ldcg(v + i)) : 0u);
+        // batches of independent loads: one block streams the whole tensor in every pass
+        for (int i0 = 0; i0 < n; i0 += nt * 8) {
+          float x[8];
+#pragma unroll
+          for (int b = 0; b < 8; ++b) {
+            const int i = i0 + b * nt + tid;
+            x[b] = i < n ? __ldcg(v + i) : 0.0f;
+          }
+#pragma unroll
+          for (int b = 0; b < 8; ++b) {
+            const bool valid = i0 + b * nt + tid < n;
+            f(valid, valid ? mag_key(x[b]) : 0u);
+          }
         }
       },
       k, 0u, 0x7FFFFFFFu, hist, sh, n_gt);
@@ -1324,7 +1332,8 @@ __device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int
   if (tid == 0) p.t_kth[j] = kth;
 }
 
-__global__ void __launch_bounds__(kEmitThreads)
+// (three blocks per SM: the rare paths may spill, the usual one must not lose occupancy)
+__global__ void __launch_bounds__(kEmitThreads, 3)
 k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
   pdl_enter();
   extern __shared__ uint32_t smask[];          // winner bitmaps of the part: [gt | eq]
