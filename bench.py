@@ -45,7 +45,7 @@ POOL = 2            # distinct pre-generated gradients per worker
 LR = 0.01
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_update_emit launch, from the ncu capture
 # summarised in profiles/k_update_emit_resnet50_ncu_full.md (same per-launch size as the bench)
-NCU_TRAFFIC_BYTES = {"resnet50": 307.19e6 + 151.20e6}
+NCU_TRAFFIC_BYTES = {"resnet50": 307.17e6 + 150.27e6}
 
 
 def _peaks():
