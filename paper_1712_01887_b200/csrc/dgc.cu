@@ -118,6 +118,9 @@ void dev_free(dgc_state* st, void* ptr) {
 // streaming pass costs 0.25 B/element flat.  The bitmap wins when more than about one entry
 // in 512 is sent.
 int defer_mask_for(double sparsity) { return (1.0 - sparsity) > 1.0 / 512.0 ? 1 : 0; }
+// Emission from v' itself (k_emit_dense) instead of from the candidate lists: from this share
+// of entries sent upwards, re-reading the part costs less than placing every candidate.
+int dense_emit_for(double sparsity) { return (1.0 - sparsity) >= kDenseEmitFraction ? 1 : 0; }
 
 // Keys one k_select block may hold in shared memory: two blocks per SM when there are more
 // tensors than SMs, else one large block.
@@ -427,6 +430,7 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   st->plan.sent_bits = st->d_sent_bits;
   if (cudaMemset(ptr, 0, (size_t)st->arena_len / 8) != cudaSuccess) return fail(DGC_ECUDA);
   st->plan.defer_mask = defer_mask_for(st->sparsity);
+  st->plan.dense_emit = dense_emit_for(st->sparsity);
   // scalars: partials[kMaxNormGrid] doubles, norm, diag[8] long long, coef, ticket, iter
   const size_t scal_bytes = (kMaxNormGrid + 1) * 8 + 8 * 8 + 16 + 8;
   if ((rc = dev_alloc(st, &ptr, scal_bytes)) != DGC_OK) return fail(rc);
@@ -475,6 +479,7 @@ int32_t dgc_set_sparsity(dgc_state* st, double sparsity) {
   rc = upload_plan(st, false);
   st->plan.sent_bits = st->d_sent_bits;
   st->plan.defer_mask = defer_mask_for(sparsity);
+  st->plan.dense_emit = dense_emit_for(sparsity);
   return rc;
 }
 
@@ -557,7 +562,8 @@ static int32_t enqueue_tail(dgc_state* st, int32_t* out_idx, float* out_val, cud
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (after_select) DGC_CUDA(cudaEventRecord(after_select, s));
-  launch(k_emit_mask, p.num_parts, kEmitThreads, kEmitSmemBytes, s, p, out_idx, out_val);
+  if (p.dense_emit) launch(k_emit_dense, p.num_parts, kEmitThreads, 0, s, p, out_idx, out_val);
+  else launch(k_emit_mask, p.num_parts, kEmitThreads, kEmitSmemBytes, s, p, out_idx, out_val);
   return check_launch();
 }
 

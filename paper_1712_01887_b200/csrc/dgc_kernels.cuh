@@ -53,6 +53,8 @@ constexpr int kEmitThreads = kPartSegs;   // one thread per segment of the part
 constexpr int kEmitRegs = 8;              // candidates per thread kept in registers
 constexpr int kMaskStride = 17;           // words per segment in the winner bitmaps (16 + 1 pad)
 constexpr int kEmitSmemBytes = 2 * kPartSegs * kMaskStride * 4;
+constexpr int kDenseChunk = 64;            // segments per chunk of k_emit_dense (128 KiB of v')
+constexpr double kDenseEmitFraction = 1.0 / 8.0;   // share of entries sent from which k_emit_dense runs
 constexpr int kMainThreads = 256;
 constexpr int kNormThreads = 256;
 constexpr int kMaxNormGrid = 2048;
@@ -134,6 +136,8 @@ struct Plan {
   // the next call's kernels zero u and v at those entries in registers before using them
   uint32_t* sent_bits;       // arena_len / 32 words, 16 per segment
   int32_t defer_mask;        // 1: masking is deferred through sent_bits
+  int32_t dense_emit;        // 1 (only with defer_mask): k_emit_dense emits from v' itself and
+                             // the candidate indices are not written
   int32_t num_tensors, num_parts, num_segs;
   int32_t num_big_parts, num_big_tensors;
 };
@@ -668,7 +672,7 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
           for (int c = 0; c < 4; ++c) {
             if (nib & (1u << c)) {
               if (pos < pm.cap) {
-                p.cand_idx[pm.cbase + pos] = e + c;
+                if (!p.dense_emit) p.cand_idx[pm.cbase + pos] = e + c;
                 p.cand_val[pm.cbase + pos] = varr[c];
               }
               ++pos;
@@ -1332,6 +1336,69 @@ __device__ void dense_select_emit(const Plan& p, const TensorMeta& t, int j, int
   if (tid == 0) p.t_kth[j] = kth;
 }
 
+// Pieces shared by the two emission kernels (block of kEmitThreads, one part per block).
+
+// Paper-literal mode: the counts vary, so the tensors' lists are packed back to back; returns
+// the first output slot of the part's tensor (what the earlier tensors send).
+__device__ __forceinline__ int emit_literal_first(const Plan& p, const PartMeta& pm, int* s_first) {
+  const int tid = threadIdx.x;
+  if (tid == 0) *s_first = 0;
+  __syncthreads();
+  int mine = 0;
+  for (int q = tid; q < pm.tensor; q += kEmitThreads) mine += __ldcg(p.t_nnz + q);
+  mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+  if ((tid & 31) == 0 && mine) atomicAdd(s_first, mine);
+  __syncthreads();
+  return *s_first;
+}
+
+// Full-selection path of a tensor (PartSel.dense == 1): its first part's block does it all.
+__device__ __forceinline__ void emit_full_selection(const Plan& p, const PartMeta& pm, int part,
+                                                    int tensor_first, int32_t* out_idx,
+                                                    float* out_val, uint32_t* smask, int* sh) {
+  const int tid = threadIdx.x;
+  __syncthreads();
+  if (tid == 0) { p.p_count[part] = 0; p.p_eq[part] = 0; }
+  if (p.defer_mask && tid < pm.nseg) {
+    // the full-selection path zeroes u and v itself: nothing is pending for this part
+    uint4* dst = reinterpret_cast<uint4*>(p.sent_bits + (size_t)(pm.seg0 + tid) * 16);
+#pragma unroll
+    for (int w = 0; w < 4; ++w) dst[w] = make_uint4(0u, 0u, 0u, 0u);
+  }
+  if (pm.first) {
+    const TensorMeta t = load_record(p.tm + pm.tensor);
+    dense_select_emit(p, t, pm.tensor, p.literal ? tensor_first : t.out_off, out_idx, out_val,
+                      smask, sh);
+  }
+}
+
+// Deferred masking: record what segment `tid` sent -- all "greater" bits and the tied bits
+// within the quota (lowest indices first); the next call zeroes u and v there.
+__device__ __forceinline__ void emit_record_sent(const Plan& p, const PartMeta& pm, int quota,
+                                                 const uint32_t* mgt, const uint32_t* meq,
+                                                 const int* s_eqb) {
+  const int tid = threadIdx.x;
+  if (tid >= pm.nseg) return;
+  int left = max(0, quota - s_eqb[tid]);
+  uint32_t words[16];
+#pragma unroll
+  for (int w = 0; w < 16; ++w) {
+    uint32_t e = meq[tid * kMaskStride + w];
+    uint32_t taken = 0;
+    while (e != 0 && left > 0) {
+      const uint32_t low = e & (0u - e);
+      taken |= low;
+      e ^= low;
+      --left;
+    }
+    words[w] = mgt[tid * kMaskStride + w] | taken;
+  }
+  uint4* dst = reinterpret_cast<uint4*>(p.sent_bits + (size_t)(pm.seg0 + tid) * 16);
+#pragma unroll
+  for (int w = 0; w < 4; ++w)
+    dst[w] = make_uint4(words[4 * w], words[4 * w + 1], words[4 * w + 2], words[4 * w + 3]);
+}
+
 // (three blocks per SM: the rare paths may spill, the usual one must not lose occupancy)
 __global__ void __launch_bounds__(kEmitThreads, 3)
 k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
@@ -1354,33 +1421,12 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   const int count = __ldcg(p.p_count + part);
   int tensor_first = 0;      // first output slot of the tensor
   if (p.literal) {
-    // paper-literal mode: the counts vary, so the tensors' lists are packed back to back:
-    // this tensor starts after what the earlier tensors send
     __shared__ int s_first;
-    if (tid == 0) s_first = 0;
-    __syncthreads();
-    int mine = 0;
-    for (int q = tid; q < pm.tensor; q += kEmitThreads) mine += __ldcg(p.t_nnz + q);
-    mine = __reduce_add_sync(0xFFFFFFFFu, mine);
-    if ((tid & 31) == 0 && mine) atomicAdd(&s_first, mine);
-    __syncthreads();
-    tensor_first = s_first;
+    tensor_first = emit_literal_first(p, pm, &s_first);
     ps.out_base += tensor_first;
   }
   if (ps.dense == 1) {
-    __syncthreads();
-    if (tid == 0) { p.p_count[part] = 0; p.p_eq[part] = 0; }
-    if (p.defer_mask && tid < pm.nseg) {
-      // the full-selection path zeroes u and v itself: nothing is pending for this part
-      uint4* dst = reinterpret_cast<uint4*>(p.sent_bits + (size_t)(pm.seg0 + tid) * 16);
-#pragma unroll
-      for (int w = 0; w < 4; ++w) dst[w] = make_uint4(0u, 0u, 0u, 0u);
-    }
-    if (pm.first) {
-      const TensorMeta t = load_record(p.tm + pm.tensor);
-      dense_select_emit(p, t, pm.tensor, p.literal ? tensor_first : t.out_off, out_idx, out_val,
-                        smask, sh);
-    }
+    emit_full_selection(p, pm, part, tensor_first, out_idx, out_val, smask, sh);
     return;
   }
   const uint32_t kth = ps.kth;
@@ -1557,27 +1603,186 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
       }
     }
   }
-  if (p.defer_mask && tid < pm.nseg) {
-    // record what was sent from segment `tid`: all "greater" bits and the tied bits within
-    // the quota (lowest indices first); the next call zeroes u and v there
-    int left = max(0, quota - s_eqb[tid]);
-    uint32_t words[16];
-#pragma unroll
-    for (int w = 0; w < 16; ++w) {
-      uint32_t e = meq[tid * kMaskStride + w];
-      uint32_t taken = 0;
-      while (e != 0 && left > 0) {
-        const uint32_t low = e & (0u - e);
-        taken |= low;
-        e ^= low;
-        --left;
-      }
-      words[w] = mgt[tid * kMaskStride + w] | taken;
+  if (p.defer_mask) emit_record_sent(p, pm, quota, mgt, meq, s_eqb);
+}
+
+// ------------------------------------------------------------------ K5b: ordered emission from v' itself
+// The same step at low sparsity (warm-up stages: a quarter of every tensor is sent).  There the
+// candidate lists are long and marking and placing each candidate costs more than reading the
+// part again, so the winners are found in v' itself -- which still holds the unmasked values,
+// because masking is deferred at these sparsities.  One warp per 512-entry segment, float4 loads
+// as in the streaming pass: a first pass counts each segment's winners, a block scan gives
+// every segment its first slot, a second pass re-reads the segment, ranks its winners with one
+// packed warp scan per 128 entries and stores the pairs in index order; the sent bits for the
+// deferred masking are assembled from the lanes' 4-bit flags by shuffles.  No bitmaps, no
+// atomics.  Candidate indices are not needed (k_update_emit does not write them in this
+// mode); the candidate values only feed the selection kernels.  Tie-fill selections need
+// nothing special here: the ties are found like every other entry.
+__global__ void __launch_bounds__(kEmitThreads, 3)
+k_emit_dense(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
+  pdl_enter();
+  __shared__ uint32_t hist[kHistWords(kEmitThreads)];   // full-selection path only
+  __shared__ int sh[66];
+  __shared__ uint32_t s_cnt[kDenseChunk];      // per segment of the chunk: winners | ties << 16
+  __shared__ uint32_t s_base[kDenseChunk + 1]; // the same before each segment; [64]: chunk total
+  const int part = blockIdx.x;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (part == 0 && tid == 0) *p.iter += 1;     // the call's last kernel counts the call
+  const PartMeta pm = load_record(p.pm + part);
+  PartSel ps = load_record(p.psel + part);
+  int tensor_first = 0;
+  if (p.literal) {
+    __shared__ int s_first;
+    tensor_first = emit_literal_first(p, pm, &s_first);
+    ps.out_base += tensor_first;
+  }
+  if (ps.dense == 1) {
+    emit_full_selection(p, pm, part, tensor_first, out_idx, out_val, hist, sh);
+    return;
+  }
+  const uint32_t kth = ps.kth;
+  const int quota = ps.quota;
+  if (tid == 0) { p.p_count[part] = 0; p.p_eq[part] = 0; }   // ready for the next call
+  const float4* v4 = reinterpret_cast<const float4*>(p.v);
+  // flags of the four entries of one float4: bits 0-3 "greater", bits 4-7 "tied"
+  auto classify = [&](const float4& x, int e) -> uint32_t {
+    const uint32_t k0 = mag_key(x.x), k1 = mag_key(x.y), k2 = mag_key(x.z), k3 = mag_key(x.w);
+    uint32_t f = (uint32_t)(k0 > kth) | (uint32_t)(k1 > kth) << 1 | (uint32_t)(k2 > kth) << 2 |
+                 (uint32_t)(k3 > kth) << 3 | (uint32_t)(k0 == kth) << 4 |
+                 (uint32_t)(k1 == kth) << 5 | (uint32_t)(k2 == kth) << 6 |
+                 (uint32_t)(k3 == kth) << 7;
+    if (e + 4 > pm.end) {                        // ragged end of the tensor
+      const int nv = max(0, pm.end - e);
+      f &= ((1u << nv) - 1u) * 0x11u;
     }
-    uint4* dst = reinterpret_cast<uint4*>(p.sent_bits + (size_t)(pm.seg0 + tid) * 16);
+    return f;
+  };
+  // The part goes through in chunks of kDenseChunk segments, so that the second pass of a chunk
+  // finds in L2 what its first pass read (the chunks of all resident blocks fit there).
+  constexpr int kWarps = kEmitThreads / 32, kPer = kDenseChunk / kWarps;
+  static_assert(kDenseChunk == 64 && kDenseChunk % kWarps == 0, "two scan warps' worth per chunk");
+  uint32_t run = 0;                                // winners | ties << 16 before the chunk ...
+  int run_g = ps.out_base, run_e = 0;              // ... unpacked and accumulated over chunks
+  for (int c0 = 0; c0 < pm.nseg; c0 += kDenseChunk) {
+    // pass 1: winners and ties of each segment of the chunk
+#pragma unroll 1
+    for (int i = 0; i < kPer; ++i) {
+      const int sgm = c0 + warp * kPer + i;
+      uint32_t cnt = 0;
+      if (sgm < pm.nseg) {
+        const int base = (pm.seg0 + sgm) * kSeg;
+        float4 x[4];
 #pragma unroll
-    for (int w = 0; w < 4; ++w)
-      dst[w] = make_uint4(words[4 * w], words[4 * w + 1], words[4 * w + 2], words[4 * w + 3]);
+        for (int r = 0; r < 4; ++r) x[r] = __ldcg(v4 + (base >> 2) + r * 32 + lane);
+        if (base + kSeg <= pm.end) {
+          // whole segment real: plain counting (the kernel is instruction-bound, not HBM-bound,
+          // unless the per-entry work stays at a few instructions)
+          int cg = 0, ce = 0;
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            const uint32_t k0 = mag_key(x[r].x), k1 = mag_key(x[r].y), k2 = mag_key(x[r].z),
+                           k3 = mag_key(x[r].w);
+            cg += (k0 > kth) + (k1 > kth) + (k2 > kth) + (k3 > kth);
+            ce += (k0 == kth) + (k1 == kth) + (k2 == kth) + (k3 == kth);
+          }
+          cnt = (uint32_t)cg | ((uint32_t)ce << 16);
+        } else {
+#pragma unroll
+          for (int r = 0; r < 4; ++r) {
+            const uint32_t f = classify(x[r], base + (r * 32 + lane) * 4);
+            cnt += (uint32_t)__popc(f & 0xFu) | ((uint32_t)__popc(f & 0xF0u) << 16);
+          }
+        }
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+      }
+      if (lane == 0) s_cnt[warp * kPer + i] = cnt;
+    }
+    __syncthreads();
+    if (warp == 0) {
+      // exclusive scan of the 64 packed counts (each half stays below 2^16: 64 x 512 entries)
+      const uint32_t a = s_cnt[lane], b2 = s_cnt[32 + lane];
+      const uint32_t ia = (uint32_t)warp_incl_scan((int)a), ib = (uint32_t)warp_incl_scan((int)b2);
+      const uint32_t ta = __shfl_sync(0xFFFFFFFFu, ia, 31);
+      s_base[lane] = ia - a;
+      s_base[32 + lane] = ta + ib - b2;
+      if (lane == 31) s_base[kDenseChunk] = ta + ib;
+    }
+    __syncthreads();
+    // pass 2: the chunk's segments in index order
+#pragma unroll 1
+    for (int i = 0; i < kPer; ++i) {
+      const int sgm = c0 + warp * kPer + i;
+      if (sgm >= pm.nseg) break;
+      const int base = (pm.seg0 + sgm) * kSeg;
+      const uint32_t sb = s_base[warp * kPer + i];
+      int lg = run_g + (int)(sb & 0xFFFFu), eqb = run_e + (int)(sb >> 16);
+      if ((s_cnt[warp * kPer + i] >> 16) == 0u && base + kSeg <= pm.end) {
+        // no ties in a whole segment (the usual case): winners only
+        lg += min(eqb, quota);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int e = base + (r * 32 + lane) * 4;
+          const float4 x = __ldcg(v4 + (e >> 2));
+          const uint32_t g = (uint32_t)(mag_key(x.x) > kth) | (uint32_t)(mag_key(x.y) > kth) << 1 |
+                             (uint32_t)(mag_key(x.z) > kth) << 2 | (uint32_t)(mag_key(x.w) > kth) << 3;
+          const int cnt = __popc(g);
+          const int incl = warp_incl_scan(cnt);
+          int pos = lg + incl - cnt;
+          if (g & 1u) { out_idx[pos] = e; out_val[pos] = x.x; ++pos; }
+          if (g & 2u) { out_idx[pos] = e + 1; out_val[pos] = x.y; ++pos; }
+          if (g & 4u) { out_idx[pos] = e + 2; out_val[pos] = x.z; ++pos; }
+          if (g & 8u) { out_idx[pos] = e + 3; out_val[pos] = x.w; }
+          uint32_t word = g << (4 * (lane & 7));
+          word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+          word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+          word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+          if ((lane & 7) == 0) p.sent_bits[(size_t)(pm.seg0 + sgm) * 16 + 4 * r + (lane >> 3)] = word;
+          lg += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        }
+        continue;
+      }
+#pragma unroll
+      for (int r = 0; r < 4; ++r) {
+        const int e = base + (r * 32 + lane) * 4;
+        const float4 x = __ldcg(v4 + (e >> 2));
+        const uint32_t f = classify(x, e);
+        const uint32_t g = f & 0xFu, q = f >> 4;
+        const int cnt = __popc(g) | (__popc(q) << 16);
+        const int incl = warp_incl_scan(cnt);
+        const int tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        const int excl = incl - cnt;
+        int pos_g = lg + (excl & 0xFFFF);          // winners before this lane's entries
+        int eb = eqb + (excl >> 16);               // ties before them, whole part
+        const float xs[4] = {x.x, x.y, x.z, x.w};
+        uint32_t took = g;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const bool gbit = (g >> c) & 1u;
+          const bool ebit = ((q >> c) & 1u) && eb < quota;   // ties: lowest indices first
+          if (gbit || ebit) {
+            const int pos = pos_g + min(eb, quota);
+            out_idx[pos] = e + c;
+            out_val[pos] = xs[c];
+          }
+          if (ebit) took |= 1u << c;
+          pos_g += gbit;
+          eb += (q >> c) & 1u;
+        }
+        // the eight lanes that share a 32-entry word put their 4-bit flags together
+        uint32_t word = took << (4 * (lane & 7));
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+        // deferred masking: sent word 4r + lane/8 of the segment
+        if ((lane & 7) == 0) p.sent_bits[(size_t)(pm.seg0 + sgm) * 16 + 4 * r + (lane >> 3)] = word;
+        lg += tot & 0xFFFF;
+        eqb += tot >> 16;
+      }
+    }
+    run = s_base[kDenseChunk];
+    run_g += (int)(run & 0xFFFFu);
+    run_e += (int)(run >> 16);
+    __syncthreads();                               // before the next chunk reuses the tables
   }
 }
 
