@@ -1717,27 +1717,39 @@ k_emit_dense(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val)
       const uint32_t sb = s_base[warp * kPer + i];
       int lg = run_g + (int)(sb & 0xFFFFu), eqb = run_e + (int)(sb >> 16);
       if ((s_cnt[warp * kPer + i] >> 16) == 0u && base + kSeg <= pm.end) {
-        // no ties in a whole segment (the usual case): winners only
+        // no ties in a whole segment (the usual case): winners only, one packed scan per two
+        // rows (a row holds at most 128 winners)
         lg += min(eqb, quota);
+#pragma unroll 1
+        for (int r0 = 0; r0 < 4; r0 += 2) {
+          float4 x[2];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int e = base + (r * 32 + lane) * 4;
-          const float4 x = __ldcg(v4 + (e >> 2));
-          const uint32_t g = (uint32_t)(mag_key(x.x) > kth) | (uint32_t)(mag_key(x.y) > kth) << 1 |
-                             (uint32_t)(mag_key(x.z) > kth) << 2 | (uint32_t)(mag_key(x.w) > kth) << 3;
-          const int cnt = __popc(g);
-          const int incl = warp_incl_scan(cnt);
-          int pos = lg + incl - cnt;
-          if (g & 1u) { out_idx[pos] = e; out_val[pos] = x.x; ++pos; }
-          if (g & 2u) { out_idx[pos] = e + 1; out_val[pos] = x.y; ++pos; }
-          if (g & 4u) { out_idx[pos] = e + 2; out_val[pos] = x.z; ++pos; }
-          if (g & 8u) { out_idx[pos] = e + 3; out_val[pos] = x.w; }
-          uint32_t word = g << (4 * (lane & 7));
-          word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
-          word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
-          word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
-          if ((lane & 7) == 0) p.sent_bits[(size_t)(pm.seg0 + sgm) * 16 + 4 * r + (lane >> 3)] = word;
-          lg += __shfl_sync(0xFFFFFFFFu, incl, 31);
+          for (int r = 0; r < 2; ++r) x[r] = __ldcg(v4 + (base >> 2) + (r0 + r) * 32 + lane);
+          uint32_t g[2];
+#pragma unroll
+          for (int r = 0; r < 2; ++r)
+            g[r] = (uint32_t)(mag_key(x[r].x) > kth) | (uint32_t)(mag_key(x[r].y) > kth) << 1 |
+                   (uint32_t)(mag_key(x[r].z) > kth) << 2 | (uint32_t)(mag_key(x[r].w) > kth) << 3;
+          const uint32_t cnt = (uint32_t)__popc(g[0]) | (uint32_t)__popc(g[1]) << 16;
+          const uint32_t incl = (uint32_t)warp_incl_scan((int)cnt);
+          const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+          const uint32_t excl = incl - cnt;
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const int e = base + ((r0 + r) * 32 + lane) * 4;
+            int pos = lg + (int)((excl >> (16 * r)) & 0xFFFFu);
+            if (g[r] & 1u) { out_idx[pos] = e; out_val[pos] = x[r].x; ++pos; }
+            if (g[r] & 2u) { out_idx[pos] = e + 1; out_val[pos] = x[r].y; ++pos; }
+            if (g[r] & 4u) { out_idx[pos] = e + 2; out_val[pos] = x[r].z; ++pos; }
+            if (g[r] & 8u) { out_idx[pos] = e + 3; out_val[pos] = x[r].w; }
+            uint32_t word = g[r] << (4 * (lane & 7));
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 1);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2);
+            word |= __shfl_xor_sync(0xFFFFFFFFu, word, 4);
+            if ((lane & 7) == 0)
+              p.sent_bits[(size_t)(pm.seg0 + sgm) * 16 + 4 * (r0 + r) + (lane >> 3)] = word;
+            lg += (int)((tot >> (16 * r)) & 0xFFFFu);
+          }
         }
         continue;
       }
