@@ -162,8 +162,13 @@ void build_host_plan(dgc_state* st, double sparsity) {
       const int64_t Q = n / 4;
       int64_t G = (int64_t)std::ceil(ratio * (double)n / 4.0);
       // a sample that holds about 1024 of the entries to send pins the proposal to +-20 %;
-      // at low sparsity that needs far fewer than ratio * n elements
-      const int64_t enough = (int64_t)std::ceil(1024.0 / std::max(1.0 - sparsity, 1e-9) / 4.0);
+      // at low sparsity that needs far fewer than ratio * n elements.  Where candidates are
+      // cheap (few entries sent) a smaller sample with a wider margin is the better trade:
+      // its rank stays within what the sampling kernel's pre-filter handles (one key per thread)
+      const double sent = std::max(1.0 - sparsity, 1e-9);
+      // (paper-literal mode keeps the one size rule that its definition states)
+      const double want = literal || sent >= 1.0 / 32.0 ? 1024.0 : sent >= 1.0 / 128.0 ? 256.0 : 128.0;
+      const int64_t enough = (int64_t)std::ceil(want / sent / 4.0);
       G = std::min<int64_t>(G, enough);
       G = std::max<int64_t>(G, 64);
       G = std::min<int64_t>(G, std::min<int64_t>(Q, kMaxSampleGroups));
