@@ -374,6 +374,12 @@ def run_ours(args):
     alg_bytes = 20.0 * total                       # read g,u,v + write u,v per real element
     achieved = alg_bytes / (k_ms * 1e-3) / 1e9
     compress_bytes = (24.0 if wl.clip_threshold > 0 else 20.0) * total + 16.0 * nnz
+    # the whole step against the same peak: every worker's compress bytes plus the receive side
+    # (lists read, dense gradient written, weights read and written; the two-call form also
+    # re-reads the dense gradient)
+    recv_bytes = 8.0 * NW * nnz + 4.0 * L + (12.0 if args.separate_receive else 8.0) * L
+    step_bytes = NW * compress_bytes + recv_bytes
+    step_gbs = step_bytes / (ms / K * 1e-3) / 1e9
     cpu = None if args.no_cpu_baseline else cpu_baseline(wl, budget_s=args.cpu_seconds)
     line = {
         "metric": METRIC, "value": whole_job_value(NW * total, K, world, ms), "unit": UNIT,
@@ -412,6 +418,8 @@ def run_ours(args):
         "compress": {"ms_per_worker": compress_ms, "elements_per_s": total / (compress_ms * 1e-3),
                      "algorithmic_gbs": compress_bytes / (compress_ms * 1e-3) / 1e9,
                      "frac_of_peak": compress_bytes / (compress_ms * 1e-3) / 1e9 / peak},
+        "step": {"algorithmic_bytes": step_bytes, "algorithmic_gbs": step_gbs,
+                 "frac_of_peak": step_gbs / peak},
         "receive": receive, "wire_format": wire, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
     }
     print(json.dumps(line))

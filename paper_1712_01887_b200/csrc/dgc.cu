@@ -263,6 +263,7 @@ int32_t upload_plan(dgc_state* st, bool first) {
   const size_t o_samp = o; o = up16(o + NS * sizeof(SampleBlock));
   const size_t o_skeys = o; o = up16(o + (size_t)st->sample_keys_total * 4);
   const size_t o_stick = o; o = up16(o + T * 4);
+  const size_t o_scnt = o; o = up16(o + NS * 4);
   const size_t NBP = st->big_parts.size(), NBT = st->big_tensors.size();
   const size_t o_bparts = o; o = up16(o + NBP * 4);
   const size_t o_btens = o; o = up16(o + NBT * 4);
@@ -304,6 +305,7 @@ int32_t upload_plan(dgc_state* st, bool first) {
   p.sample_blocks = (const SampleBlock*)(d + o_samp);
   p.sample_keys = (uint32_t*)(d + o_skeys);
   p.sample_ticket = (int32_t*)(d + o_stick);
+  p.sample_cnt = (int32_t*)(d + o_scnt);
   p.big_parts = (const int32_t*)(d + o_bparts);
   p.big_tensors = (const int32_t*)(d + o_btens);
   p.big_hist = (int32_t*)(d + o_bhist);

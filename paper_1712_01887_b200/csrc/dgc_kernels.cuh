@@ -111,6 +111,7 @@ struct Plan {
   const SampleBlock* sample_blocks;
   uint32_t* sample_keys;     // |v'| keys of the current call's sample, all tensors
   int32_t* sample_ticket;    // per tensor: sampling blocks that have finished
+  int32_t* sample_cnt;       // per sampling block: keys it kept in its slice of sample_keys
   // multi-block selection (tensors with too many candidates for one block)
   const int32_t* big_parts;  // parts of the big tensors
   const int32_t* big_tensors;
@@ -417,6 +418,8 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   const TensorMeta t = load_record(p.tm + j);
   const int G = t.groups, rank = t.rank;
   uint4* gkeys = reinterpret_cast<uint4*>(p.sample_keys + t.key_base);
+  uint4 mykeys = make_uint4(0u, 0u, 0u, 0u);
+  bool have = false;
   {
     const int s = sb.chunk * kSampleThreads + tid;
     if (s < G) {
@@ -442,8 +445,55 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
       mc_step<CLIP, NEST>(gg.y, coef, m, u.y, v.y);
       mc_step<CLIP, NEST>(gg.z, coef, m, u.z, v.z);
       mc_step<CLIP, NEST>(gg.w, coef, m, u.w, v.w);
-      gkeys[s] = make_uint4(mag_key(v.x), mag_key(v.y), mag_key(v.z), mag_key(v.w));
+      mykeys = make_uint4(mag_key(v.x), mag_key(v.y), mag_key(v.z), mag_key(v.w));
+      have = true;
     }
+  }
+  // Tensors sampled by several blocks: every block keeps only the keys that can be among the
+  // tensor's `rank` largest -- its own `rank` largest (and their ties), zeros never -- and
+  // writes them packed into its slice; the last block then selects among a few thousand keys
+  // instead of re-reading the whole sample.  (If fewer than `rank` keys of the sample are
+  // non-zero the union is short and the answer is 0.)
+  const bool local = t.chunks > 1 && rank <= kSampleThreads;   // (larger ranks: tiny samples)
+  if (local) {
+    uint32_t* slice = p.sample_keys + t.key_base + sb.chunk * (4 * kSampleThreads);
+    const int nv = min(kSampleThreads, G - sb.chunk * kSampleThreads);   // threads with a group
+    const uint32_t tmax = have ? max(max(mykeys.x, mykeys.y), max(mykeys.z, mykeys.w)) : 0u;
+    if (tid == 0) { s_cnt = 0; s_max = 0u; }
+    __syncthreads();
+    uint32_t low = 1u;                             // zeros are never kept: see the union below
+    if (rank <= 4 * nv) {
+      const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
+      if (lane == 0) atomicMax(&s_max, wmax);
+      __syncthreads();
+      int n_gt_local;
+      low = max(1u, block_select_desc<kSampleThreads, false>(
+                        [&](auto f) {
+                          f(have, mykeys.x);
+                          f(have, mykeys.y);
+                          f(have, mykeys.z);
+                          f(have, mykeys.w);
+                        },
+                        rank, 0u, s_max, hist, sh, n_gt_local));
+    }
+    const uint32_t karr[4] = {mykeys.x, mykeys.y, mykeys.z, mykeys.w};
+    if (__any_sync(0xFFFFFFFFu, have && tmax >= low)) {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const bool keep = have && karr[c] >= low;
+        const unsigned mk = __ballot_sync(0xFFFFFFFFu, keep);
+        if (mk) {
+          int basepos = 0;
+          if (lane == __ffs(mk) - 1) basepos = atomicAdd(&s_cnt, __popc(mk));
+          basepos = __shfl_sync(0xFFFFFFFFu, basepos, __ffs(mk) - 1);
+          if (keep) slice[basepos + __popc(mk & ((1u << lane) - 1u))] = karr[c];
+        }
+      }
+    }
+    __syncthreads();
+    if (tid == 0) p.sample_cnt[blockIdx.x] = s_cnt;
+  } else if (have) {
+    gkeys[sb.chunk * kSampleThreads + tid] = mykeys;
   }
   if (t.chunks > 1) {
     __threadfence();
@@ -457,10 +507,68 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
     if (!s_last) return;
     __threadfence();
   }
-  if (tid == 0) { s_cnt = 0; s_max = 0u; }
+  int n_gt, n_eq = 0;
+  uint32_t kth = 0;
+  bool done = false;
+  if (local) {
+    // the union of the blocks' slices: counts -> offsets (at most 32 blocks per tensor)
+    __shared__ int s_off[33];
+    static_assert(kMaxSampleGroups <= 32 * kSampleThreads, "one warp scans the blocks' counts");
+    const int first = blockIdx.x - sb.chunk;
+    if (tid == 0) s_max = 0u;
+    if (tid < 32) {
+      const int c = tid < t.chunks ? __ldcg(p.sample_cnt + first + tid) : 0;
+      const int incl = warp_incl_scan(c);
+      s_off[tid] = incl - c;
+      if (tid == 31) s_off[32] = incl;
+    }
+    __syncthreads();
+    const int U = s_off[32];
+    const uint32_t* keys0 = p.sample_keys + t.key_base;
+    if (U < rank) {
+      kth = 0u;                                    // fewer than `rank` non-zero keys
+      n_eq = 2;                                    // and the zeros beyond them are many
+    } else if (U <= kSampleSurvivors) {
+      uint32_t tmax = 0u;
+      for (int q = tid >> 5; q < t.chunks; q += kSampleThreads / 32) {
+        const int o = s_off[q], c = s_off[q + 1] - o;
+        const uint32_t* src = keys0 + q * (4 * kSampleThreads);
+        for (int i = lane; i < c; i += 32) {
+          const uint32_t key = __ldcg(src + i);
+          surv[o + i] = key;
+          tmax = max(tmax, key);
+        }
+      }
+      const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
+      if (lane == 0) atomicMax(&s_max, wmax);
+      __syncthreads();
+      const int it2 = (U + kSampleThreads - 1) / kSampleThreads;
+      kth = block_select_desc<kSampleThreads, false>(
+          [&](auto f) {
+            for (int it = 0; it < it2; ++it) {
+              const int i = it * kSampleThreads + tid;
+              f(i < U, i < U ? surv[i] : 0u);
+            }
+          },
+          rank, 0u, s_max, hist, sh, n_gt, &n_eq);
+    } else {
+      kth = block_select_desc<kSampleThreads>(
+          [&](auto f) {
+            // one warp per slice: the warps' loads run side by side
+            for (int q = tid >> 5; q < t.chunks; q += kSampleThreads / 32) {
+              const int c = s_off[q + 1] - s_off[q];
+              const uint32_t* src = keys0 + q * (4 * kSampleThreads);
+              for (int i = lane; i < c; i += 32) f(true, __ldcg(src + i));
+            }
+          },
+          rank, 0u, 0x7FFFFFFFu, hist, sh, n_gt, &n_eq);
+    }
+    done = true;
+  }
+  if (tid == 0 && !done) { s_cnt = 0; s_max = 0u; }
   __syncthreads();                                    // also orders this block's own key writes
-  // this block now holds the whole sample of the tensor in gkeys[0 .. G)
-  const int iters = (G + kSampleThreads - 1) / kSampleThreads;
+  // (otherwise) this block now holds the whole sample of the tensor in gkeys[0 .. G)
+  const int iters = done ? 0 : (G + kSampleThreads - 1) / kSampleThreads;
   uint32_t tmax = 0;
 #pragma unroll 4
   for (int it = 0; it < iters; ++it) {
@@ -477,10 +585,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   __syncthreads();
   const uint32_t kmax = s_max;
   const int owners = min(G, kSampleThreads);          // threads that hold at least one group
-  int n_gt, n_eq = 0;
-  uint32_t kth = 0;
-  bool done = false;
-  if (rank <= owners) {
+  if (!done && rank <= owners) {
     // lower bound: rank-th largest of the thread maxima
     const uint32_t low = block_select_desc<kSampleThreads, false>([&](auto f) { f(tid < owners, tmax); }, rank, 0u, kmax,
                                            hist, sh, n_gt);
