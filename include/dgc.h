@@ -82,7 +82,8 @@ typedef struct dgc_status {
   double  grad_norm;          /* L2 norm of the last gradient set (0 when clipping is off)   */
   float   clip_coef;          /* coefficient applied to the last gradient (1 = not clipped)  */
   int32_t flags;              /* OR of DGC_FLAG_* over the last dgc_compress                 */
-  int64_t iterations;         /* dgc_compress calls so far                                   */
+  int64_t iterations;         /* dgc_compress calls completed on the device (graph replays   */
+                              /* included)                                                   */
   int64_t full_select_last;   /* tensors that took the full-selection path in the last call */
   int64_t candidates_last;    /* entries that passed the sampled thresholds in the last call */
 } dgc_status;
