@@ -159,13 +159,13 @@ def test_all_zero_gradient_is_zero_filled_with_lowest_indices(P):
     pair.close()
 
 
-@pytest.mark.parametrize("sparsity", [0.999, 0.99])
+@pytest.mark.parametrize("sparsity", [0.999, 0.99, 0.75])
 def test_fewer_nonzeros_than_k_zero_fill_matches_oracle(P, sparsity):
     """Tensors with fewer non-zero entries than k (an almost unused embedding, a frozen layer):
     all non-zeros plus the lowest-index zeros, over several iterations with momentum so that u
     is non-zero where v was sent.  Covers one-part, multi-part and (at 99 %) multi-block-selected
-    tensors, a ragged last segment, immediate (99.9 %) and deferred (99 %) masking, and zeros
-    of either sign."""
+    tensors, a ragged last segment, immediate (99.9 %) and deferred (99 %) masking, emission
+    from v' itself (75 %), and zeros of either sign."""
     numel = [700001, 1 << 22, 40000, 300, 1 << 19]
     pair = P.Pair(numel, 1, 0.9, 0.0, sparsity, seed=4)
     rep = P.ParityReport()
@@ -198,7 +198,7 @@ def test_fewer_nonzeros_than_k_zero_fill_matches_oracle(P, sparsity):
     pair.close()
 
 
-@pytest.mark.parametrize("sparsity", [0.999, 0.99])
+@pytest.mark.parametrize("sparsity", [0.999, 0.99, 0.75])
 def test_few_distinct_magnitudes_tie_fill_matches_oracle(P, sparsity):
     """Sign-like gradients: every entry of a tensor has one of a handful of magnitudes, so the
     k-th largest |v| is shared by far more than k entries.  Those ties are counted, not listed
