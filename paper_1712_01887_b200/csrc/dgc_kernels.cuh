@@ -1609,12 +1609,18 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
     }
     __syncthreads();
   }
-  // thread s owns segment s: popcounts, then winners before each segment
+  // thread s owns segment s: popcounts (the count of the segment's first eight words goes to
+  // its padding word), then winners before each segment
+  bool has_eq;
   {
     int gt = 0, eq = 0;
     if (tid < pm.nseg) {
 #pragma unroll
       for (int w = 0; w < 16; ++w) {
+        if (w == 8) {
+          mgt[tid * kMaskStride + 16] = (uint32_t)gt;
+          meq[tid * kMaskStride + 16] = (uint32_t)eq;
+        }
         gt += __popc(mgt[tid * kMaskStride + w]);
         eq += __popc(meq[tid * kMaskStride + w]);
       }
@@ -1623,16 +1629,21 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
     block_excl_scan2(gt, eq, sh, bg, be, tg, te);
     s_gtb[tid] = bg;
     s_eqb[tid] = be;
+    has_eq = te > 0;                             // hardly ever: then the tie counts are skipped
   }
   __syncthreads();
   auto emit = [&](int local, float val, uint32_t key) {
     const int s = local >> 9, w = (local >> 5) & 15;
     const uint32_t below = (1u << (local & 31)) - 1u;
-    int lg = __popc(mgt[s * kMaskStride + w] & below);
-    int le = __popc(meq[s * kMaskStride + w] & below);
-    for (int x = 0; x < w; ++x) {
-      lg += __popc(mgt[s * kMaskStride + x]);
-      le += __popc(meq[s * kMaskStride + x]);
+    const uint32_t* mg = mgt + s * kMaskStride;
+    const int x0 = w & 8;                        // words before x0 are in the padding word's count
+    int lg = __popc(mg[w] & below) + (x0 ? (int)mg[16] : 0);
+    for (int x = x0; x < w; ++x) lg += __popc(mg[x]);
+    int le = 0;
+    if (has_eq) {
+      const uint32_t* me = meq + s * kMaskStride;
+      le = __popc(me[w] & below) + (x0 ? (int)me[16] : 0);
+      for (int x = x0; x < w; ++x) le += __popc(me[x]);
     }
     const int eq_before = s_eqb[s] + le;         // ties with a lower index, whole part
     int pos;
