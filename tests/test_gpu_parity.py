@@ -791,3 +791,45 @@ def test_checkpoint_resume_paper_literal_needs_the_call_count(P):
         b.set_iterations(-1)
     a.close()
     b.close()
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_randomised_shapes_distributions_and_sparsities(P, case):
+    """Seeded fuzz over what the selection paths branch on: tensor sizes around the segment,
+    part and sampling boundaries, sparsities on both sides of the deferred-masking and
+    emission-from-v' switches, clipping and Nesterov on or off, and value distributions with
+    heavy tails, exact zeros, few distinct magnitudes or constants.  Three iterations each,
+    bit for bit against the oracle; the slow full-selection path must never be needed."""
+    rng = np.random.default_rng(1000 + case)
+    pool = [1, 3, 31, 512, 513, 4095, 8192, 8193, 20000, 70001, 262144, 262145, 300000,
+            524288 + 7, 1 << 20, (1 << 21) + 5, 3000000]
+    numel = [int(x) for x in rng.choice(pool, size=int(rng.integers(2, 6)))]
+    if case % 3 == 0:
+        numel.append(int(rng.choice([1 << 22, 5000000])))       # multi-block selection at low s
+    sparsity = float(rng.choice([0.0, 0.5, 0.75, 0.9, 0.9375, 0.99, 0.996, 0.999, 0.9999]))
+    clip = float(rng.choice([0.0, 1.0]))
+    nest = bool(rng.integers(0, 2))
+    pair = P.Pair(numel, 4, 0.9, clip, sparsity, seed=int(rng.integers(1, 1 << 30)), nesterov=nest)
+    rep = P.ParityReport()
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    kinds = ["normal", "student", "sparse", "levels", "const", "zero"]
+    for t in range(3):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for o, n in zip(off, numel):
+            kind = kinds[int(rng.integers(0, len(kinds)))]
+            if kind == "normal":
+                x = rng.standard_normal(n)
+            elif kind == "student":
+                x = rng.standard_t(3, size=n) * 1e-4
+            elif kind == "sparse":
+                x = rng.standard_normal(n) * (rng.random(n) < 0.003)
+            elif kind == "levels":
+                x = rng.integers(-2, 3, size=n) * 0.125
+            elif kind == "const":
+                x = np.full(n, 0.5) * (rng.integers(0, 2, size=n) * 2 - 1)
+            else:
+                x = np.zeros(n)
+            g[o:o + n] = x.astype(np.float32)
+        _, _, st = pair.step(g, rep, check_state=(t == 2))
+        assert st.full_select_last == 0, (case, t, numel, sparsity, st.flags)
+    pair.close()
