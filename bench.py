@@ -226,6 +226,8 @@ def run_ours(args):
         step(t)
     barrier()
     graphs, graph_launches = None, 0
+    graphs_used = bool(args.graph)
+    eager_step = step
     if args.graph:
         # the whole step captured once per pooled gradient and replayed: every replay is one
         # more iteration on the same buffers (the library keeps its per-call state on the device)
@@ -237,7 +239,6 @@ def run_ours(args):
                 step(i)
             graph_launches = B.launch_count() - n0
             graphs.append(gr)
-        eager_step = step
 
         def step(t):                               # noqa: F811
             graphs[t % POOL].replay()
@@ -374,6 +375,32 @@ def run_ours(args):
     alg_bytes = 20.0 * total                       # read g,u,v + write u,v per real element
     achieved = alg_bytes / (k_ms * 1e-3) / 1e9
     compress_bytes = (24.0 if wl.clip_threshold > 0 else 20.0) * total + 16.0 * nnz
+    # optional: where on the GPU's clock each worker's kernels ran in one step (the library's
+    # timeline aid: first and last block start of every kernel), with the GPU kept busy while
+    # the host enqueues the step so that the step runs as it does in the timed loop
+    timeline = None
+    if args.timeline:
+        for s_ in states:
+            s_.timeline_enable(True)
+        for t in range(3):
+            eager_step(t) if graphs_used else step(t)
+        torch.cuda.synchronize()
+        for s_ in states:
+            s_.timeline_read()
+        busy = torch.empty(1 << 28, dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            busy.zero_()
+        (eager_step if graphs_used else step)(3)
+        torch.cuda.synchronize()
+        tl = np.stack([s_.timeline_read().astype(np.int64) for s_ in states])      # [NW, 4, 2]
+        t0 = tl[:, :, 0][tl[:, :, 1] > 0].min()
+        timeline = {"unit": "us after the step's first block",
+                    "kernels": ["sample", "stream", "select", "emit"],
+                    "first_last_block_start": [[[round(float(x - t0) / 1e3, 1) for x in k]
+                                                for k in w] for w in tl]}
+        for s_ in states:
+            s_.timeline_enable(False)
+        del busy
     # the whole step against the same peak: every worker's compress bytes plus the receive side
     # (lists read, dense gradient written, weights read and written; the two-call form also
     # re-reads the dense gradient)
@@ -420,6 +447,7 @@ def run_ours(args):
                      "frac_of_peak": compress_bytes / (compress_ms * 1e-3) / 1e9 / peak},
         "step": {"algorithmic_bytes": step_bytes, "algorithmic_gbs": step_gbs,
                  "frac_of_peak": step_gbs / peak},
+        "timeline": timeline,
         "receive": receive, "wire_format": wire, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
     }
     print(json.dumps(line))
@@ -651,6 +679,9 @@ def main():
     ap.add_argument("--flush-l2", action="store_true",
                     help="rewrite a 256 MB buffer before every timed step (cold L2) and sum "
                          "per-step event times")
+    ap.add_argument("--timeline", action="store_true",
+                    help="add the GPU-clock timeline of one step (per worker and kernel: first "
+                         "and last block start) to the JSON line")
     ap.add_argument("--graph", action="store_true",
                     help="capture the step into CUDA graphs (one per pooled gradient) and time "
                          "their replays")

@@ -317,6 +317,20 @@ int32_t dgc_state_set_iterations(dgc_state* st, int64_t iterations, void* stream
 int32_t dgc_profile_enable(dgc_state* st, int32_t max_calls);
 int32_t dgc_profile_read(dgc_state* st, float* ms_out, int32_t capacity, int32_t* count_out);
 
+/* Measurement aid (not part of the method): where on the GPU's clock the kernels of this
+ * state's calls ran, also when several states' calls overlap on different streams (which
+ * events on one stream cannot show).  While enabled, every block of the sampling, streaming,
+ * selection and emission kernels notes its start on the GPU's nanosecond timer.
+ * dgc_timeline_read synchronises `stream` and returns, since the last read (or enable),
+ *   ns_out[2 * kernel]      the earliest block start
+ *   ns_out[2 * kernel + 1]  the latest block start
+ * for kernel 0 sampling, 1 streaming pass, 2 selection, 3 emission (UINT64_MAX / 0 if the
+ * kernel did not run), then clears them.  Differences between states on one GPU are
+ * meaningful; the origin is arbitrary.  dgc_timeline_enable synchronises the device;
+ * DGC_EINVAL from dgc_timeline_read if not enabled. */
+int32_t dgc_timeline_enable(dgc_state* st, int32_t on);
+int32_t dgc_timeline_read(dgc_state* st, void* stream, uint64_t* ns_out);
+
 /* Number of kernels this library has launched in this process (all states). */
 uint64_t dgc_launch_count(void);
 

@@ -87,6 +87,8 @@ _sigs = {
     "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_write": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_set_iterations": (ctypes.c_int32, [_vp, ctypes.c_int64, _vp]),
+    "dgc_timeline_enable": (ctypes.c_int32, [_vp, ctypes.c_int32]),
+    "dgc_timeline_read": (ctypes.c_int32, [_vp, _vp, _vp]),
     "dgc_profile_enable": (ctypes.c_int32, [_vp, ctypes.c_int32]),
     "dgc_profile_read": (ctypes.c_int32, [_vp, _vp, ctypes.c_int32,
                                           ctypes.POINTER(ctypes.c_int32)]),
@@ -246,6 +248,16 @@ class State:
         _check(_lib.dgc_state_write(self._h, None if u is None else u.ctypes.data,
                                     None if v is None else v.ctypes.data, _stream(stream)),
                "dgc_state_write")
+
+    def timeline_enable(self, on: bool = True) -> None:
+        _check(_lib.dgc_timeline_enable(self._h, int(bool(on))), "dgc_timeline_enable")
+
+    def timeline_read(self, stream=None) -> np.ndarray:
+        """[4 kernels][first block start, last block start] in ns of the GPU timer."""
+        out = np.zeros(8, np.uint64)
+        _check(_lib.dgc_timeline_read(self._h, _stream(stream), out.ctypes.data),
+               "dgc_timeline_read")
+        return out.reshape(4, 2)
 
     def set_iterations(self, iterations: int, stream=None) -> None:
         _check(_lib.dgc_state_set_iterations(self._h, int(iterations), _stream(stream)),

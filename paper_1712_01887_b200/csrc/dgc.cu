@@ -83,6 +83,7 @@ struct dgc_state {
   int prof_cap = 0, prof_n = 0;
   int norm_grid = 0;
   int select_smem_keys = 0;
+  unsigned long long* d_timeline = nullptr;
   bool alive = false;
 };
 
@@ -902,6 +903,36 @@ int32_t dgc_get_thresholds(dgc_state* st, void* stream, uint32_t* kth_key, int32
   if (kth_key) DGC_CUDA(cudaMemcpy(kth_key, st->plan.t_kth, T * 4, cudaMemcpyDeviceToHost));
   if (candidates) DGC_CUDA(cudaMemcpy(candidates, st->plan.t_cand, T * 4, cudaMemcpyDeviceToHost));
   return DGC_OK;
+}
+
+static int32_t timeline_reset(dgc_state* st) {
+  unsigned long long init[8];
+  for (int i = 0; i < 4; ++i) { init[2 * i] = ~0ull; init[2 * i + 1] = 0ull; }
+  DGC_CUDA(cudaMemcpy(st->d_timeline, init, sizeof init, cudaMemcpyHostToDevice));
+  return DGC_OK;
+}
+
+int32_t dgc_timeline_enable(dgc_state* st, int32_t on) {
+  if (!st || !st->alive) return DGC_ESTATE;
+  DGC_CUDA(cudaSetDevice(st->device));
+  DGC_CUDA(cudaDeviceSynchronize());
+  if (on && !st->d_timeline) {
+    void* ptr = nullptr;
+    const int32_t rc = dev_alloc(st, &ptr, 64);
+    if (rc != DGC_OK) return rc;
+    st->d_timeline = (unsigned long long*)ptr;
+  }
+  st->plan.timeline = on ? st->d_timeline : nullptr;
+  return on ? timeline_reset(st) : DGC_OK;
+}
+
+int32_t dgc_timeline_read(dgc_state* st, void* stream, uint64_t* ns_out) {
+  if (!st || !st->alive) return DGC_ESTATE;
+  if (!ns_out) return DGC_EINVAL;
+  if (!st->plan.timeline) return DGC_EINVAL;
+  DGC_CUDA(cudaStreamSynchronize(as_stream(stream)));
+  DGC_CUDA(cudaMemcpy(ns_out, st->d_timeline, 64, cudaMemcpyDeviceToHost));
+  return timeline_reset(st);
 }
 
 int32_t dgc_profile_enable(dgc_state* st, int32_t max_calls) {

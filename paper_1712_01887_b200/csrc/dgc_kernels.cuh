@@ -137,6 +137,9 @@ struct Plan {
   // the next call's kernels zero u and v at those entries in registers before using them
   uint32_t* sent_bits;       // arena_len / 32 words, 16 per segment
   int32_t defer_mask;        // 1: masking is deferred through sent_bits
+  unsigned long long* timeline;   // measurement aid, NULL = off: per kernel of the call (sampling,
+                             // streaming, selection, emission) the earliest and the latest
+                             // block start on the GPU's nanosecond timer
   int32_t dense_emit;        // 1 (only with defer_mask): k_emit_dense emits from v' itself and
                              // the candidate indices are not written
   int32_t num_tensors, num_parts, num_segs;
@@ -165,6 +168,16 @@ __device__ __forceinline__ T load_record(const T* ptr) {
 // 10 % slower steps with early signalling).  The wait is executed by every block, so that
 // "grid N has completed" still implies "grid N-1 has completed".
 __device__ __forceinline__ void pdl_enter() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Timeline aid: every block of the four kernels of a compress call notes when it started.
+__device__ __forceinline__ void timeline_mark(unsigned long long* tl, int kernel) {
+  if (tl != nullptr && threadIdx.x == 0) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    atomicMin(tl + 2 * kernel, t);
+    atomicMax(tl + 2 * kernel + 1, t);
+  }
+}
 
 __device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
 
@@ -405,6 +418,7 @@ template <bool CLIP, bool NEST>
 __global__ void __launch_bounds__(kSampleThreads)
 k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_base) {
   pdl_enter();
+  timeline_mark(p.timeline, 0);
   const uint64_t call_seed = seed_base + (uint64_t)__ldcg(p.iter);
   __shared__ uint32_t hist[kHistWords(kSampleThreads)];
   __shared__ uint32_t surv[kSampleSurvivors];
@@ -663,6 +677,7 @@ template <bool CLIP, bool NEST>
 __global__ void __launch_bounds__(kMainThreads)
 k_update_emit(Plan p, const float* __restrict__ g, float m) {
   pdl_enter();
+  timeline_mark(p.timeline, 1);
   const int lane = threadIdx.x & 31;
   const float4* g4 = reinterpret_cast<const float4*>(g);
   float4* u4 = reinterpret_cast<float4*>(p.u);
@@ -842,6 +857,7 @@ __device__ __forceinline__ bool tie_fill_parts(const Plan& p, int p0, int pn, in
 __global__ void __launch_bounds__(kSelectThreads)
 k_select(Plan p, int smem_keys) {
   pdl_enter();
+  timeline_mark(p.timeline, 2);
   const int parity = (int)(__ldcg(p.iter) & 1);
   extern __shared__ uint32_t dyn_smem[];          // [histograms | keys]
   uint32_t* hist = dyn_smem;
@@ -1508,6 +1524,7 @@ __device__ __forceinline__ void emit_record_sent(const Plan& p, const PartMeta& 
 __global__ void __launch_bounds__(kEmitThreads, 3)
 k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
   pdl_enter();
+  timeline_mark(p.timeline, 3);
   extern __shared__ uint32_t smask[];          // winner bitmaps of the part: [gt | eq]
   __shared__ int sh[66];
   __shared__ int s_gtb[kPartSegs];             // winners before each segment
@@ -1737,6 +1754,7 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
 __global__ void __launch_bounds__(kEmitThreads, 3)
 k_emit_dense(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) {
   pdl_enter();
+  timeline_mark(p.timeline, 3);
   __shared__ uint32_t hist[kHistWords(kEmitThreads)];   // full-selection path only
   __shared__ int sh[66];
   __shared__ uint32_t s_cnt[kDenseChunk];      // per segment of the chunk: winners | ties << 16

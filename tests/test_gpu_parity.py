@@ -833,3 +833,36 @@ def test_randomised_shapes_distributions_and_sparsities(P, case):
         _, _, st = pair.step(g, rep, check_state=(t == 2))
         assert st.full_select_last == 0, (case, t, numel, sparsity, st.flags)
     pair.close()
+
+
+def test_timeline_aid_orders_the_kernels_of_a_call(P):
+    """dgc_timeline_*: block start times on the GPU clock, per kernel of a compress call.  The
+    results of the call do not change; the kernels appear in the order the algorithm needs."""
+    from paper_1712_01887_b200 import binding as B
+    numel = [300000, 5000, 70001]
+    rng = np.random.default_rng(5)
+    a = B.State(numel, 1, 0.9, 0.0, 0.999, seed=3)
+    b = B.State(numel, 1, 0.9, 0.0, 0.999, seed=3)
+    L = a.arena_len
+    g = torch.from_numpy(rng.standard_normal(L).astype(np.float32)).cuda()
+    oa = (torch.empty(a.max_nnz, dtype=torch.int32, device="cuda"),
+          torch.empty(a.max_nnz, dtype=torch.float32, device="cuda"))
+    ob = (torch.empty_like(oa[0]), torch.empty_like(oa[1]))
+    with pytest.raises(B.DgcError):
+        a.timeline_read()                        # not enabled
+    a.timeline_enable(True)
+    a.compress(g, *oa)
+    b.compress(g, *ob)
+    tl = a.timeline_read().astype(np.int64)
+    assert (tl[:, 0] <= tl[:, 1]).all() and (tl[:, 0] > 0).all()
+    assert tl[0, 0] <= tl[1, 0] <= tl[2, 0] <= tl[3, 0]          # sample, stream, select, emit
+    assert tl[0, 1] <= tl[1, 0] and tl[1, 1] <= tl[2, 0] and tl[2, 1] <= tl[3, 0]
+    assert torch.equal(oa[0], ob[0]) and torch.equal(oa[1].view(torch.int32), ob[1].view(torch.int32))
+    empty = a.timeline_read()
+    assert (empty[:, 1] == 0).all() and (empty[:, 0] == np.iinfo(np.uint64).max).all()
+    a.timeline_enable(False)
+    a.compress(g, *oa)
+    with pytest.raises(B.DgcError):
+        a.timeline_read()
+    a.close()
+    b.close()
