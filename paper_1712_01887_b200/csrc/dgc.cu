@@ -332,8 +332,11 @@ int32_t upload_plan(dgc_state* st, bool first) {
   int keys = (int)std::min<int64_t>(st->max_tensor_expect, select_key_cap(st));
   keys = std::max(keys, 1024);
   st->select_smem_keys = keys;
-  DGC_CUDA(cudaFuncSetAttribute(k_select, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (keys + kHistWords(kSelectThreads)) * 4));
+  // (the attribute is per function, not per state: always the largest any state may ask for)
+  DGC_CUDA(cudaFuncSetAttribute(k_select<kSelectThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (kSelectMaxSmemKeys + kHistWords(kSelectThreads)) * 4));
+  DGC_CUDA(cudaFuncSetAttribute(k_select<kSelectBatchThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (kSelectMaxSmemKeys + kHistWords(kSelectBatchThreads)) * 4));
   return DGC_OK;
 }
 
@@ -553,11 +556,17 @@ static int32_t enqueue_stream_pass(dgc_state* st, const float* grad_arena, cudaS
 }
 
 static int32_t enqueue_tail(dgc_state* st, int32_t* out_idx, float* out_val, cudaStream_t s,
-                            cudaEvent_t after_select = nullptr) {
+                            cudaEvent_t after_select = nullptr, bool batch = false) {
   const Plan& p = st->plan;
   int32_t rc;
-  launch(k_select, p.num_tensors, kSelectThreads,
-         (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s, p, st->select_smem_keys);
+  if (batch)
+    launch(k_select<kSelectBatchThreads>, p.num_tensors, kSelectBatchThreads,
+           (size_t)(st->select_smem_keys + kHistWords(kSelectBatchThreads)) * 4, s, p,
+           st->select_smem_keys);
+  else
+    launch(k_select<kSelectThreads>, p.num_tensors, kSelectThreads,
+           (size_t)(st->select_smem_keys + kHistWords(kSelectThreads)) * 4, s, p,
+           st->select_smem_keys);
   if ((rc = check_launch()) != DGC_OK) return rc;
   if (p.num_big_parts > 0) {
     launch(k_big_hist<0>, p.num_big_parts, kBigThreads, 0, s, p);
@@ -652,7 +661,7 @@ int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
     dgc_state* st = states[w];
     if ((rc = enqueue_head(st, grad_arenas[w], q, nullptr)) != DGC_OK) return rc;
     if ((rc = enqueue_stream_pass(st, grad_arenas[w], q)) != DGC_OK) return rc;
-    if ((rc = enqueue_tail(st, out_idx[w], out_val[w], q)) != DGC_OK) return rc;
+    if ((rc = enqueue_tail(st, out_idx[w], out_val[w], q, nullptr, num_states >= 4)) != DGC_OK) return rc;
     st->iterations += 1;
   }
   for (int i = 0; i < used; ++i) {

@@ -47,6 +47,7 @@ constexpr int kMaxSampleGroups = 16384; // float4 groups sampled per tensor at m
 constexpr int kSampleThreads = 512;    // one sampled float4 group per thread and block
 constexpr int kSampleSurvivors = 4096;
 constexpr int kSelectThreads = 1024;
+constexpr int kSelectBatchThreads = 512;   // k_select in a batch of several workers
 constexpr int kSelectMaxSmemKeys = 51200;
 constexpr int kSelectMaxParts = 256;   // parts of one tensor whose tables fit in shared memory
 constexpr int kEmitThreads = kPartSegs;   // one thread per segment of the part
@@ -817,18 +818,19 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
 // This is the path of a tensor that is all or almost all zeros (a frozen layer, unused
 // embedding rows: the key is 0) or holds a few distinct magnitudes (sign or low-bit
 // gradients).  Returns false, having written nothing, if the ties do not suffice.
+template <int THREADS>
 __device__ __forceinline__ bool tie_fill_parts(const Plan& p, int p0, int pn, int k, int total,
                                                int out_off, uint32_t kth, int* sh) {
   const int tid = threadIdx.x;
   int mine = 0;
-  for (int q = tid; q < pn; q += kSelectThreads) mine += __ldcg(p.p_eq + p0 + q);
+  for (int q = tid; q < pn; q += THREADS) mine += __ldcg(p.p_eq + p0 + q);
   int e1, e2, eq_total, t2;
   block_excl_scan2(mine, 0, sh, e1, e2, eq_total, t2);
   __syncthreads();
   if (total + eq_total < k) return false;
   const int quota = k - total;
   int run_gt = 0, run_eq = 0;
-  for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+  for (int q0 = 0; q0 < pn; q0 += THREADS) {
     const int q = q0 + tid;
     int gt = 0, eq = 0;
     if (q < pn) {
@@ -854,14 +856,18 @@ __device__ __forceinline__ bool tie_fill_parts(const Plan& p, int p0, int pn, in
   return true;
 }
 
-__global__ void __launch_bounds__(kSelectThreads)
+// THREADS: 1024 for a call that runs alone (shortest chain for the largest tensor), 512 when
+// several workers' selections run together (twice the blocks per SM: the batch's tail is
+// bound by block slots, not by one block's chain).
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
 k_select(Plan p, int smem_keys) {
   pdl_enter();
   timeline_mark(p.timeline, 2);
   const int parity = (int)(__ldcg(p.iter) & 1);
   extern __shared__ uint32_t dyn_smem[];          // [histograms | keys]
   uint32_t* hist = dyn_smem;
-  uint32_t* skeys = dyn_smem + kHistWords(kSelectThreads);
+  uint32_t* skeys = dyn_smem + kHistWords(THREADS);
   __shared__ int sh[66];
   __shared__ int s_flag;
   __shared__ uint32_t s_max;
@@ -896,7 +902,7 @@ k_select(Plan p, int smem_keys) {
     __syncthreads();
     total = s_pbase[pn];
   } else {
-    for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+    for (int q0 = 0; q0 < pn; q0 += THREADS) {
       const int q = q0 + tid;
       int c = 0;
       if (q < pn) {
@@ -925,7 +931,7 @@ k_select(Plan p, int smem_keys) {
   const int rank = lit_own ? k + 1 : k;
   if (!overflow && !literal && total < k && t.groups > 0) {
     const uint32_t tie_key = __ldcg(p.p_thr + p0) - 1u;
-    if (tie_fill_parts(p, p0, pn, k, total, t.out_off, tie_key, sh)) {
+    if (tie_fill_parts<THREADS>(p, p0, pn, k, total, t.out_off, tie_key, sh)) {
       if (tid == 0) {
         p.t_kth[j] = tie_key;
         p.t_cand[j] = total;
@@ -939,7 +945,7 @@ k_select(Plan p, int smem_keys) {
   if (overflow || (!literal && total < k)) {
     if (tid == 0) p.t_nnz[j] = k;
     // full-selection path: k_emit_mask's block of the tensor's first part does it
-    for (int q = tid; q < pn; q += kSelectThreads) {
+    for (int q = tid; q < pn; q += THREADS) {
       PartSel ps;
       ps.kth = 0u; ps.quota = 0; ps.out_base = 0; ps.dense = 1;
       p.psel[p0 + q] = ps;
@@ -954,14 +960,14 @@ k_select(Plan p, int smem_keys) {
     return;
   }
   const bool in_smem = tables && total <= smem_keys;
-  const int slices = max(1, (kSelectThreads / 32) / pn);
+  const int slices = max(1, (THREADS / 32) / pn);
   uint32_t kmax = 0x7FFFFFFFu;
   uint32_t kbase = 0u;
   if (in_smem) {
     // gather the keys of all parts, compact, into shared memory: coalesced reads, a part is
     // shared by `slices` warps when the tensor has fewer parts than the block has warps
     uint32_t tmax = 0;
-    for (int unit = warp; unit < pn * slices; unit += kSelectThreads / 32) {
+    for (int unit = warp; unit < pn * slices; unit += THREADS / 32) {
       const int q = unit / slices, sl = unit - q * slices;
       const int b0 = s_pbase[q], c = s_pbase[q + 1] - b0;
       const float* src = p.cand_val + s_pcb[q];
@@ -987,28 +993,28 @@ k_select(Plan p, int smem_keys) {
     kth = 0u;                                    // k = n: everything, zeros included
     n_gt = 0;
   } else if (in_smem) {
-    const int iters = (total + kSelectThreads - 1) / kSelectThreads;
+    const int iters = (total + THREADS - 1) / THREADS;
     auto each = [&](auto f) {
       for (int it = 0; it < iters; ++it) {
-        const int i = it * kSelectThreads + tid;
+        const int i = it * THREADS + tid;
         const bool valid = i < total;
         f(valid, valid ? skeys[i] : kbase);
       }
     };
     // up to two keys per thread: not worth private histograms
-    if (total <= 2 * kSelectThreads)
-      kth = block_select_desc<kSelectThreads, false>(each, rank, kbase, kmax, hist, sh, n_gt);
+    if (total <= 2 * THREADS)
+      kth = block_select_desc<THREADS, false>(each, rank, kbase, kmax, hist, sh, n_gt);
     else
-      kth = block_select_desc<kSelectThreads, true>(each, rank, kbase, kmax, hist, sh, n_gt);
+      kth = block_select_desc<THREADS, true>(each, rank, kbase, kmax, hist, sh, n_gt);
   } else {
-    kth = block_select_desc<kSelectThreads>(
+    kth = block_select_desc<THREADS>(
         [&](auto f) {
           for (int q = 0; q < pn; ++q) {
             const int c = __ldcg(p.p_count + p0 + q);
             const float* src = p.cand_val + __ldg(&p.pm[p0 + q].cbase);
-            const int iters = (c + kSelectThreads - 1) / kSelectThreads;
+            const int iters = (c + THREADS - 1) / THREADS;
             for (int it = 0; it < iters; ++it) {
-              const int i = it * kSelectThreads + tid;
+              const int i = it * THREADS + tid;
               const bool valid = i < c;
               f(valid, valid ? mag_key(__ldcg(src + i)) : 0u);
             }
@@ -1023,10 +1029,10 @@ k_select(Plan p, int smem_keys) {
   if (tables) {
     // per part: strictly-greater and tied candidates (a single part needs no count: it takes
     // the whole quota and k_emit_mask stops at the quota by itself)
-    for (int q = tid; q < pn; q += kSelectThreads) { s_gt[q] = 0; s_eq[q] = 0; }
+    for (int q = tid; q < pn; q += THREADS) { s_gt[q] = 0; s_eq[q] = 0; }
     __syncthreads();
     if (pn > 1) {
-      for (int unit = warp; unit < pn * slices; unit += kSelectThreads / 32) {
+      for (int unit = warp; unit < pn * slices; unit += THREADS / 32) {
         const int q = unit / slices, sl = unit - q * slices;
         const int b0 = s_pbase[q], c = s_pbase[q + 1] - b0;
         const float* src = p.cand_val + s_pcb[q];
@@ -1062,7 +1068,7 @@ k_select(Plan p, int smem_keys) {
       }
     } else {
       int run_gt = 0, run_eq = 0;
-      for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+      for (int q0 = 0; q0 < pn; q0 += THREADS) {
         const int q = q0 + tid;
         const int gt = q < pn ? s_gt[q] : 0, eq = q < pn ? s_eq[q] : 0;
         int bg, be, tg, te;
@@ -1085,7 +1091,7 @@ k_select(Plan p, int smem_keys) {
   } else {
     // more parts than the tables hold: walk them in chunks, counting from global memory
     int run_gt = 0, run_eq = 0;
-    for (int q0 = 0; q0 < pn; q0 += kSelectThreads) {
+    for (int q0 = 0; q0 < pn; q0 += THREADS) {
       const int q = q0 + tid;
       int gt = 0, eq = 0;
       if (q < pn) {
@@ -1291,7 +1297,7 @@ k_big_final(Plan p) {
   bool tie_fill = false;
   if (overflow == 0 && !literal && total < k) {
     kth = __ldcg(p.p_thr + p0) - 1u;
-    tie_fill = tie_fill_parts(p, p0, pn, k, total, t.out_off, kth, sh);
+    tie_fill = tie_fill_parts<kSelectThreads>(p, p0, pn, k, total, t.out_off, kth, sh);
   }
   const bool dense = !tie_fill && (overflow != 0 || (!literal && total < k));
   // paper-literal mode: at most 2k passed the sampled threshold -> all of them are sent
