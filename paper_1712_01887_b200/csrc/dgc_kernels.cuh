@@ -1568,7 +1568,11 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
     const int i = b * kEmitThreads + tid;
     vals[b] = i < count ? __ldcg(cval + i) : 0.0f;
   }
-  for (int i = tid; i < 2 * kPartSegs * kMaskStride; i += kEmitThreads) smask[i] = 0u;
+  // (only the part's own segments: most parts of a many-tensor set are a few segments long)
+  for (int i = tid; i < pm.nseg * kMaskStride; i += kEmitThreads) {
+    mgt[i] = 0u;
+    meq[i] = 0u;
+  }
   __syncthreads();
   if (tid == 0) { p.p_count[part] = 0; p.p_eq[part] = 0; }   // ready for the next call
   // mark the candidates that reach the threshold: one bit per element of the part
