@@ -6,6 +6,8 @@ import os
 import subprocess
 import sys
 
+import pytest
+
 import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
@@ -65,3 +67,31 @@ def test_reference_arm_prints_contract_line_and_other_ranks_stay_silent():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
     assert line["config"]["workload"] == "lstm_small"
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("flags", [[], ["--graph", "--timeline"], ["--flush-l2", "--no-batch"],
+                                   ["--separate-receive", "--timeline"]])
+def test_bench_options_print_the_contract_line(flags):
+    """The benchmark's own arm on the small L2-resident case with its optional modes: one JSON
+    line with the contract's keys, launches counted, a roofline object, and the timeline when
+    asked for."""
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    cmd = [sys.executable, os.path.join(root, "bench.py"), "--workload", "cfg1", "--steps", "4",
+           "--warmup", "3", "--no-e2e", "--no-cpu-baseline"] + flags
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=600, cwd=root)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    for key in ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step",
+                "higher_is_better", "scaling", "dtype", "data", "config", "roofline",
+                "gpu_launches", "clocks"):
+        assert key in line, key
+    assert line["steps"] == 4 and line["value"] > 0 and line["gpu_launches"] > 0
+    assert line["roofline"]["bound"] == "hbm" and 0 < line["roofline"]["frac"] < 2
+    if "--timeline" in flags:
+        tl = line["timeline"]["first_last_block_start"]
+        assert len(tl) == line["config"]["simulated_workers"] and len(tl[0]) == 4
+        for w in tl:
+            assert w[0][0] <= w[1][0] <= w[2][0] <= w[3][0]
+    else:
+        assert line["timeline"] is None
