@@ -32,7 +32,10 @@
 //
 // Pins (tests/test_oracle_*.py): hand-worked dyadic traces, brute-force full
 // sort for n <= 4096, closed forms of Eq. 4/5, conservation, s = 0 reducing to
-// plain synchronous SGD, numpy's float64 norm, numpy's stable argsort.
+// plain synchronous SGD, numpy's float64 norm, numpy's stable argsort; for the
+// Sec. 5 selection: numpy partition on hand-chosen sample positions (rank
+// k_s against k_s +- 1, ties at the threshold, 2k against 2k + 1 passing) and
+// the published SplitMix64 outputs for the position generator.
 
 #include <algorithm>
 #include <cmath>
@@ -224,8 +227,8 @@ void dgc_oracle_apply_sgd(float* w, const float* dense_grad, int64_t len, float 
   }
 }
 
-// Sec. 3.1: "The encode() function packs the 32-bit nonzero gradient values and 16-bit
-// run lengths of zeros."  Entry t = (run_t, value_t): run_t zeros are skipped, then value_t
+// Sec. 3.1, encode(): the wire format is 32-bit values plus 16-bit zero run lengths.
+// Entry t = (run_t, value_t): run_t zeros are skipped, then value_t
 // is stored.  The paper gives no rule for more than 65535 zeros in a row; the reading used
 // here bridges the gap with filler entries (65535, +0.0f), each standing for 65535 zeros
 // followed by one slot that holds an explicit zero.  Zeros after the last entry are not
@@ -270,18 +273,67 @@ int64_t dgc_oracle_decode_runlength(const uint16_t* runs, const float* values, i
 }
 
 // ---------------------------------------------------------------------------------------
-// The sampled selection as Sec. 5 states it ("paper-literal" mode): the threshold is taken
-// from a sample and applied to the whole tensor; only "if the number of gradients exceeding
-// the threshold is far more than expected, a precise threshold is calculated from the
-// already-selected gradients".  The number of entries sent then varies.  Readings (the paper
-// gives none of these): the sample is one group of 4 consecutive elements per stratum at a
-// hashed position (below); thr is the k_s-th largest sampled |v|, k_s = ceil(S (1 - s)), so
-// that "|v| > thr" keeps n k_s / (S + 1) ~ n (1 - s) entries on average; "far more" = more
-// than 2 k_j, in which case the exact top-k_j is sent; tensors of <= 8192 elements are their
-// own sample, and for them thr is the (k_j + 1)-th largest |v| (the largest entry not to be
-// sent), so that "|v| > thr" keeps the top k_j minus whatever ties with thr.  The positions come from a counter-based hash that this
-// file and the CUDA library each implement.
+// The sampled selection as Sec. 5 states it ("paper-literal" mode).  Sec. 5 in short: draw a
+// sample of 0.1 % to 1 % of the tensor, take the top-k threshold of the sample as the threshold
+// of the whole tensor, and only when far more entries than expected pass it, select precisely
+// among those that passed.  The number of entries sent then varies from call to call.
+//
+// Readings (Sec. 5 gives no numbers beyond the 0.1 % .. 1 % range):
+//   * sample size   S = ceil(rho n_j), rho the configured sample ratio (integer arithmetic in
+//                   parts per 1e9, like k_j; at least 1, at most n_j); every tensor is sampled
+//   * positions     S independent uniform draws from [0, n_j), with replacement; they are an
+//                   INPUT of the selection below (the draws come from the counter-based
+//                   generator further down, which holds no arithmetic of the method)
+//   * threshold     thr = the k_s-th largest sampled |v|, k_s = ceil(S (1 - s)) (the top-k
+//                   selection of Alg. 4 applied to the sample, same integer k formula)
+//   * mask          |v| > thr over the whole tensor (Alg. 4's strict compare)
+//   * "far more than expected" = more than 2 k_j entries pass; then exactly the top k_j of the
+//                   tensor are sent (all of them passed, so this is the precise selection
+//                   among the already-selected entries; ties go to the lower index)
+//   * fewer than k_j pass (also none): what passed is sent as it is
 
+// S = ceil(rho n), at least 1, at most n (rho <= 0 selects the default 1 %).
+int64_t dgc_oracle_sample_count(int64_t n, double sample_ratio) {
+  const double ratio = sample_ratio > 0.0 ? sample_ratio : 0.01;
+  const long long q = std::llround(ratio * 1e9);
+  long long S = (static_cast<long long>(n) * q + 999999999LL) / 1000000000LL;
+  if (S < 1) S = 1;
+  if (S > n) S = n;
+  return S;
+}
+
+// Selection of one tensor from an explicit sample.  v: the n accumulated values (already
+// updated); positions[0..S): the sampled indices, each in [0, n), repeats allowed and counted
+// as separate draws.  Returns the number of entries chosen, their indices ascending in sel_idx
+// (room for min(n, 2k)).  thr_key_out (may be NULL) receives the threshold's bit pattern.
+int64_t dgc_oracle_select_from_sample(int64_t n, const float* v, const int64_t* positions,
+                                      int64_t S, int64_t k, double sparsity, int64_t* sel_idx,
+                                      uint32_t* thr_key_out) {
+  // top-k_s of the sample -> threshold
+  std::vector<uint32_t> sample(static_cast<size_t>(S));
+  for (int64_t r = 0; r < S; ++r) sample[static_cast<size_t>(r)] = magnitude_key(v[positions[r]]);
+  const int64_t ks = dgc_oracle_topk_count(S, sparsity);
+  std::sort(sample.begin(), sample.end(), std::greater<uint32_t>());
+  const uint32_t thr = sample[static_cast<size_t>(ks - 1)];
+  if (thr_key_out) *thr_key_out = thr;
+  // mask of the whole tensor
+  int64_t passed = 0;
+  for (int64_t i = 0; i < n; ++i) passed += magnitude_key(v[i]) > thr;
+  if (passed > 2 * k) {
+    // far more than expected: the precise top-k_j
+    dgc_oracle_select_topk(n, v, k, sel_idx, 0);
+    return k;
+  }
+  int64_t c = 0;
+  for (int64_t i = 0; i < n; ++i)
+    if (magnitude_key(v[i]) > thr) sel_idx[c++] = i;
+  return c;
+}
+
+// Counter-based generator of the sample positions (no arithmetic of the method): draw r of
+// tensor j in a call is floor(h n / 2^64) with h = mix(call_seed xor (j << 32) xor r), mix =
+// the SplitMix64 step (add the golden-ratio increment, then its two multiply-xorshift rounds).
+// The CUDA library implements the same generator on its side.
 static inline uint64_t oracle_mix64(uint64_t x) {
   x += 0x9E3779B97F4A7C15ull;
   x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
@@ -289,69 +341,24 @@ static inline uint64_t oracle_mix64(uint64_t x) {
   return x ^ (x >> 31);
 }
 
-// Groups of 4 elements sampled from a tensor of n elements (0: the whole tensor is the sample).
-int64_t dgc_oracle_sample_groups(int64_t n, double sparsity, double sample_ratio) {
-  if (n <= 8192) return 0;
-  const double ratio = sample_ratio > 0.0 ? sample_ratio : 0.01;
-  long long G = (long long)std::ceil(ratio * (double)n / 4.0);
-  const long long enough = (long long)std::ceil(1024.0 / std::max(1.0 - sparsity, 1e-9) / 4.0);
-  G = std::min(G, enough);
-  G = std::max(G, 64LL);
-  G = std::min(G, std::min((long long)(n / 4), 16384LL));
-  return G;
+uint64_t dgc_oracle_mix64(uint64_t x) { return oracle_mix64(x); }
+
+void dgc_oracle_sample_positions(int64_t n, int64_t S, uint64_t call_seed, int32_t tensor_index,
+                                 int64_t* positions) {
+  for (int64_t r = 0; r < S; ++r) {
+    const uint64_t h = oracle_mix64(call_seed ^
+                                    (static_cast<uint64_t>(static_cast<uint32_t>(tensor_index)) << 32) ^
+                                    static_cast<uint64_t>(r));
+    positions[r] = static_cast<int64_t>(
+        (static_cast<unsigned __int128>(h) * static_cast<unsigned __int128>(n)) >> 64);
+  }
 }
 
-// Selection of one tensor in paper-literal mode.  v: the n accumulated values (already
-// updated).  Returns the number of entries chosen; their local indices ascending in sel_idx
-// (capacity min(n, 2k)).
-int64_t dgc_oracle_select_sampled(int64_t n, const float* v, int64_t k, double sparsity,
-                                  double sample_ratio, uint64_t call_seed, int32_t tensor_index,
-                                  int64_t* sel_idx) {
-  const int64_t G = dgc_oracle_sample_groups(n, sparsity, sample_ratio);
-  std::vector<uint32_t> sample;
-  if (G == 0) {
-    sample.resize(static_cast<size_t>(n));
-    for (int64_t i = 0; i < n; ++i) sample[static_cast<size_t>(i)] = magnitude_key(v[i]);
-  } else {
-    const uint32_t W = static_cast<uint32_t>((n / 4) / G);        // groups per stratum
-    sample.reserve(static_cast<size_t>(4 * G));
-    for (int64_t st = 0; st < G; ++st) {
-      const uint32_t h = static_cast<uint32_t>(oracle_mix64(
-          call_seed ^ (static_cast<uint64_t>(static_cast<uint32_t>(tensor_index)) << 32) ^
-          static_cast<uint64_t>(static_cast<uint32_t>(st))));
-      const uint64_t grp = static_cast<uint64_t>(st) * W +
-                           ((static_cast<uint64_t>(h) * static_cast<uint64_t>(W)) >> 32);
-      for (int c = 0; c < 4; ++c) sample.push_back(magnitude_key(v[4 * grp + c]));
-    }
-  }
-  const int64_t S = static_cast<int64_t>(sample.size());
-  const int64_t ks = dgc_oracle_topk_count(S, sparsity);
-  // rank of thr in the sample: k_s for a true sample, k + 1 when the tensor is its own sample;
-  // no threshold at all if that rank does not exist (everything is to be sent)
-  const int64_t rank = G == 0 ? k + 1 : ks;
-  bool have_thr = rank <= S;
-  uint32_t thr = 0;
-  if (have_thr) {
-    std::nth_element(sample.begin(), sample.begin() + (rank - 1), sample.end(),
-                     std::greater<uint32_t>());
-    thr = sample[static_cast<size_t>(rank - 1)];
-  }
-  std::vector<int64_t> pass;
-  for (int64_t i = 0; i < n; ++i)
-    if (!have_thr || magnitude_key(v[i]) > thr) pass.push_back(i);
-  if (static_cast<int64_t>(pass.size()) > 2 * k) {
-    // far more than expected: the precise top-k_j (same order as everywhere: ties to the lower index)
-    dgc_oracle_select_topk(n, v, k, sel_idx, 0);
-    return k;
-  }
-  for (size_t r = 0; r < pass.size(); ++r) sel_idx[r] = pass[r];
-  return static_cast<int64_t>(pass.size());
-}
-
-// One iteration in paper-literal mode: clip, momentum correction, then per tensor the
-// sampled selection above, emission and masking.  The pairs of all tensors are packed back to
+// One iteration in paper-literal mode: clip, momentum correction, then per tensor the sample
+// positions of this call, the selection from that sample, emission and masking.  The pairs of all tensors are packed back to
 // back (tensor order, ascending index); nnz_out[j] = entries sent from tensor j.
-// seed/iteration give call_seed = seed * 0x9E3779B97F4A7C15 + iteration (mod 2^64).
+// seed/iteration give call_seed = mix(seed * 0x9E3779B97F4A7C15 + iteration) (mod 2^64), so
+// that consecutive calls draw unrelated positions.
 int64_t dgc_oracle_compress_sampled(int32_t num_tensors, const int64_t* offset,
                                     const int64_t* numel, const int64_t* k, float* u, float* v,
                                     const float* g, float momentum, double clip_threshold,
@@ -367,14 +374,18 @@ int64_t dgc_oracle_compress_sampled(int32_t num_tensors, const int64_t* offset,
   *norm_out = norm;
   *coef_out = coef;
   dgc_oracle_momentum_correction(num_tensors, offset, numel, u, v, g, momentum, coef, nesterov);
-  const uint64_t call_seed = seed * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(iteration);
-  std::vector<int64_t> sel;
+  const uint64_t call_seed =
+      oracle_mix64(seed * 0x9E3779B97F4A7C15ull + static_cast<uint64_t>(iteration));
+  std::vector<int64_t> sel, pos;
   int64_t out = 0;
   for (int32_t j = 0; j < num_tensors; ++j) {
     const int64_t o = offset[j];
     sel.assign(static_cast<size_t>(std::min(numel[j], 2 * k[j])), 0);
-    const int64_t c = dgc_oracle_select_sampled(numel[j], v + o, k[j], sparsity, sample_ratio,
-                                                call_seed, j, sel.data());
+    const int64_t S = dgc_oracle_sample_count(numel[j], sample_ratio);
+    pos.assign(static_cast<size_t>(S), 0);
+    dgc_oracle_sample_positions(numel[j], S, call_seed, j, pos.data());
+    const int64_t c = dgc_oracle_select_from_sample(numel[j], v + o, pos.data(), S, k[j], sparsity,
+                                                    sel.data(), nullptr);
     nnz_out[j] = c;
     for (int64_t r = 0; r < c; ++r) {
       const int64_t i = o + sel[static_cast<size_t>(r)];

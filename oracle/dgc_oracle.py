@@ -65,8 +65,17 @@ def lib() -> ctypes.CDLL:
                                                    ctypes.c_int64]
         L.dgc_oracle_apply_sgd.restype = None
         L.dgc_oracle_apply_sgd.argtypes = [_f32p, _f32p, ctypes.c_int64, ctypes.c_float]
-        L.dgc_oracle_sample_groups.restype = ctypes.c_int64
-        L.dgc_oracle_sample_groups.argtypes = [ctypes.c_int64, ctypes.c_double, ctypes.c_double]
+        L.dgc_oracle_sample_count.restype = ctypes.c_int64
+        L.dgc_oracle_sample_count.argtypes = [ctypes.c_int64, ctypes.c_double]
+        L.dgc_oracle_mix64.restype = ctypes.c_uint64
+        L.dgc_oracle_mix64.argtypes = [ctypes.c_uint64]
+        L.dgc_oracle_sample_positions.restype = None
+        L.dgc_oracle_sample_positions.argtypes = [ctypes.c_int64, ctypes.c_int64, ctypes.c_uint64,
+                                                  ctypes.c_int32, _i64p]
+        L.dgc_oracle_select_from_sample.restype = ctypes.c_int64
+        L.dgc_oracle_select_from_sample.argtypes = [ctypes.c_int64, _f32p, _i64p, ctypes.c_int64,
+                                                    ctypes.c_int64, ctypes.c_double, _i64p,
+                                                    ctypes.POINTER(ctypes.c_uint32)]
         L.dgc_oracle_compress_sampled.restype = ctypes.c_int64
         L.dgc_oracle_compress_sampled.argtypes = [
             ctypes.c_int32, _i64p, _i64p, _i64p, _f32p, _f32p, _f32p, ctypes.c_float,
@@ -184,8 +193,40 @@ class Worker:
         return CompressResult(idx, val, norm.value, np.float32(coef.value))
 
 
-def sample_groups(n: int, sparsity: float, sample_ratio: float = 0.01) -> int:
-    return int(lib().dgc_oracle_sample_groups(int(n), float(sparsity), float(sample_ratio)))
+def sample_count(n: int, sample_ratio: float = 0.01) -> int:
+    """Sec. 5: size of the sample of a tensor of n elements, ceil(ratio * n)."""
+    return int(lib().dgc_oracle_sample_count(int(n), float(sample_ratio)))
+
+
+def mix64(x: int) -> int:
+    return int(lib().dgc_oracle_mix64(ctypes.c_uint64(int(x) & 0xFFFFFFFFFFFFFFFF)))
+
+
+def call_seed(seed: int, iteration: int) -> int:
+    """Seed of the sample positions of one call (state seed, calls completed before it)."""
+    return mix64((int(seed) * 0x9E3779B97F4A7C15 + int(iteration)) & 0xFFFFFFFFFFFFFFFF)
+
+
+def sample_positions(n: int, count: int, seed: int, tensor_index: int) -> np.ndarray:
+    """The `count` sample positions of tensor `tensor_index` for the call seed `seed`."""
+    pos = np.empty(int(count), dtype=np.int64)
+    lib().dgc_oracle_sample_positions(int(n), int(count), ctypes.c_uint64(int(seed)),
+                                      int(tensor_index), _p(pos, _i64p))
+    return pos
+
+
+def select_from_sample(v: np.ndarray, positions: np.ndarray, k: int, sparsity: float):
+    """Sec. 5 selection of one tensor from an explicit sample: (chosen indices ascending,
+    bit pattern of the threshold)."""
+    v = _chk(v, np.float32)
+    positions = _chk(np.ascontiguousarray(positions), np.int64)
+    assert positions.size >= 1 and positions.min() >= 0 and positions.max() < v.size
+    sel = np.empty(min(v.size, 2 * int(k)), dtype=np.int64)
+    thr = ctypes.c_uint32()
+    c = lib().dgc_oracle_select_from_sample(v.size, _p(v, _f32p), _p(positions, _i64p),
+                                            positions.size, int(k), float(sparsity),
+                                            _p(sel, _i64p), ctypes.byref(thr))
+    return sel[:c].copy(), int(thr.value)
 
 
 def compress_sampled(worker: "Worker", g: np.ndarray, seed: int, iteration: int,

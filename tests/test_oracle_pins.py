@@ -461,68 +461,189 @@ def test_encode_runlength_round_trip_and_size():
 
 
 # ------------------------------------------------------------------ paper-literal sampled selection (Sec. 5)
+# The selection takes the sample positions as an input, so it is pinned here on positions
+# chosen by hand, against numpy's partition of |v| at those positions; the position generator
+# is pinned separately against the published SplitMix64 outputs.
 
 def _numpy_topk_set(v, k):
     return set(_numpy_topk(v, k).tolist())
 
 
-def test_sampled_selection_small_tensor_is_its_own_sample():
-    """n <= 8192: the sample is the tensor, thr is the (k+1)-th largest |v|, "|v| > thr" keeps
-    the top k minus whatever ties with thr: checked against numpy's sort."""
-    rng = np.random.default_rng(41)
-    for n, s in ((1000, 0.99), (8192, 0.999), (64, 0.75), (5, 0.0)):
-        w = O.Worker([0], [n], n, 1, 0.0, 0.0, s)
-        g = rng.standard_normal(n).astype(np.float32)
-        r, nnz = O.compress_sampled(w, g.copy(), seed=1, iteration=0)
-        k = O.topk_count(n, s)
-        if k == n:
-            expect = np.arange(n)
-        else:
-            a = np.abs(g)
-            thr = np.sort(a)[::-1][k]
-            expect = np.flatnonzero(a > thr)
-        assert r.idx.tolist() == expect.tolist() and nnz.tolist() == [expect.size]
-        assert r.val.tobytes() == g[expect].tobytes()
-    # ties with the (k+1)-th are not sent
-    w = O.Worker([0], [8], 8, 1, 0.0, 0.0, 0.75)      # k = 2
-    r, nnz = O.compress_sampled(w, _f32([5, 3, 3, 3, 1, 0, 0, 0]), seed=0, iteration=0)
-    assert r.idx.tolist() == [0] and nnz.tolist() == [1]
+def _numpy_from_sample(v, positions, k, sparsity):
+    """Sec. 5 with numpy: threshold = the ceil(S (1 - s))-th largest sampled |v| (np.partition),
+    mask |v| > thr, exact top-k when more than 2k pass."""
+    a = np.abs(v)
+    samp = a[np.asarray(positions)]
+    S = samp.size
+    ks = max(1, -((-S * round((1 - sparsity) * 10**9)) // 10**9))      # ceil in integers
+    thr = np.partition(samp, S - ks)[S - ks]
+    passed = np.flatnonzero(a > thr)
+    if passed.size > 2 * k:
+        return _numpy_topk(v, k), thr
+    return passed, thr
 
 
-def test_sampled_selection_threshold_is_a_sample_quantile():
-    """Large iid tensors: what passes is a superset or subset of the exact top-k with a count
-    near k (the sample holds k_s = 40 of the entries to send), every sent entry dominates every
-    unsent one, and nothing beyond 2k is ever sent."""
-    rng = np.random.default_rng(43)
-    n, s = 400000, 0.99
+def test_sample_threshold_rank_is_ceil_S_times_1_minus_s():
+    """Distinct magnitudes 1..n at known places: the sample's sorted values are known, so the
+    threshold is readable by eye, and rank k_s - 1 or k_s + 1 would give another count."""
+    n = 1000
+    v = _f32(np.arange(1, n + 1))                         # |v_i| = i + 1
+    v[::2] *= -1                                          # signs must not matter
+    # S = 20 positions holding the values 50, 100, ..., 1000; s = 0.9 -> k_s = ceil(2.0) = 2
+    positions = np.arange(49, n, 50)
+    sel, thr = O.select_from_sample(v, positions, k=500, sparsity=0.9)
+    assert np.array([thr], np.uint32).view(np.float32)[0] == 950.0    # 2nd largest of the sample
+    assert sel.tolist() == list(range(950, 1000))         # the 50 values above 950, ascending
+    # S(1-s) an exact integer must not be rounded up by a float ceil: s = 0.75, S = 20 -> 5
+    sel, thr = O.select_from_sample(v, positions, k=500, sparsity=0.75)
+    assert np.array([thr], np.uint32).view(np.float32)[0] == 800.0
+    assert sel.size == 200
+    # s = 0.999 -> k_s = ceil(0.02) = 1: the sample maximum; nothing exceeds 1000 -> nothing sent
+    sel, thr = O.select_from_sample(v, positions, k=500, sparsity=0.999)
+    assert np.array([thr], np.uint32).view(np.float32)[0] == 1000.0 and sel.size == 0
+    # s = 0.94 -> S(1-s) = 1.2 -> k_s = 2 (ceil, not round)
+    sel, thr = O.select_from_sample(v, positions, k=500, sparsity=0.94)
+    assert np.array([thr], np.uint32).view(np.float32)[0] == 950.0
+    # order of the positions is irrelevant, a repeated position counts as two draws
+    sel2, thr2 = O.select_from_sample(v, positions[::-1].copy(), k=500, sparsity=0.9)
+    assert sel2.tolist() == list(range(950, 1000)) and thr2 == thr
+    rep = np.concatenate([positions, [999]])              # 1000 drawn twice: S = 21, k_s = 3
+    sel3, thr3 = O.select_from_sample(v, rep, k=500, sparsity=0.9)
+    assert np.array([thr3], np.uint32).view(np.float32)[0] == 950.0   # 1000, 1000, 950
+    assert sel3.tolist() == list(range(950, 1000))
+
+
+def test_sample_threshold_ties_and_strict_compare():
+    """Entries equal to the threshold are not sent (strict >), also when the sample holds the
+    threshold value several times."""
+    v = _f32([5, 3, 3, 3, 1, 0, 7, 3, 9, 2])
+    # sample = {3, 3, 9, 1}: s = 0.5 -> k_s = 2 -> thr = 3 -> sent: 5, 7, 9
+    sel, thr = O.select_from_sample(v, np.array([1, 2, 8, 4]), k=4, sparsity=0.5)
+    assert np.array([thr], np.uint32).view(np.float32)[0] == 3.0
+    assert sel.tolist() == [0, 6, 8]
+    # threshold 0 (sample of zeros): every non-zero passes; 8 > 2k = 4 -> exact top-2 = {8, 6}
+    sel, thr = O.select_from_sample(v, np.array([5, 5, 5]), k=2, sparsity=0.5)
+    assert thr == 0 and sel.tolist() == [6, 8]
+
+
+def test_far_more_than_expected_is_more_than_2k():
+    """Exactly 2k passing entries are sent as they are; 2k + 1 trigger the precise top-k."""
+    n = 100
+    v = _f32(np.arange(n))                                # |v_i| = i
+    # sample {89}: thr = 89 -> 10 entries pass (90..99)
+    sel, _ = O.select_from_sample(v, np.array([89]), k=5, sparsity=0.9)     # 10 == 2k
+    assert sel.tolist() == list(range(90, 100))
+    sel, _ = O.select_from_sample(v, np.array([88]), k=5, sparsity=0.9)     # 11 > 2k
+    assert sel.tolist() == list(range(95, 100))
+    # and the precise selection keeps the tie rule (lower index first)
+    v = _f32([4, 4, 4, 4, 4, 4, 1, 0])
+    sel, _ = O.select_from_sample(v, np.array([6]), k=2, sparsity=0.5)      # 6 pass > 4
+    assert sel.tolist() == [0, 1]
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_selection_from_sample_matches_numpy_partition(seed):
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(50, 20000))
+    s = float(rng.choice([0.5, 0.9, 0.99, 0.999]))
+    v = rng.standard_t(3, n).astype(np.float32)
+    if seed % 2:
+        v = np.round(v * 4) / 4                           # many exact ties
+        v = v.astype(np.float32)
+    S = int(rng.integers(1, max(2, n // 10)))
+    positions = rng.integers(0, n, S)
     k = O.topk_count(n, s)
-    assert O.sample_groups(n, s) == 1000            # 1% of n / 4, below the other caps
-    counts = []
-    for it in range(6):
-        w = O.Worker([0], [n], n, 1, 0.0, 0.0, s)
-        g = rng.standard_normal(n).astype(np.float32)
-        r, nnz = O.compress_sampled(w, g.copy(), seed=7, iteration=it)
-        c = int(nnz[0])
-        counts.append(c)
-        assert 0.4 * k < c < 1.8 * k              # 40 of the 4000 sampled lie above thr: +-16 %
-        sent = np.zeros(n, bool)
-        sent[r.idx] = True
-        assert np.abs(g[sent]).min() > np.abs(g[~sent]).max()
-        top = _numpy_topk_set(g, k)
-        got = set(r.idx.tolist())
-        assert got <= top or top <= got
-        assert not w.u[r.idx].any() and not w.v[r.idx].any()
-    assert len(set(counts)) > 1                       # the count really varies with the sample
+    sel, thr = O.select_from_sample(v, positions, k, s)
+    ref, thr_ref = _numpy_from_sample(v, positions, k, s)
+    assert np.array([thr], np.uint32).view(np.float32)[0] == thr_ref
+    assert sel.tolist() == ref.tolist()
 
 
-def test_sampled_selection_far_more_than_expected_gives_exact_topk():
+def test_sample_size_is_the_configured_share_of_the_tensor():
+    """Sec. 5: 0.1 % to 1 % of the gradients; ceil, at least one, never more than n."""
+    assert O.sample_count(400000, 0.01) == 4000
+    assert O.sample_count(400001, 0.01) == 4001
+    assert O.sample_count(1 << 28, 0.01) == 2684355       # no cap: still 1 % of 2^28
+    assert O.sample_count(1 << 28, 0.001) == 268436
+    assert O.sample_count(64, 0.01) == 1
+    assert O.sample_count(1, 0.01) == 1
+    assert O.sample_count(3, 0.5) == 2
+    assert O.sample_count(1000, 0.0) == 10                # 0 selects the default 1 %
+
+
+def test_position_generator_is_splitmix64_scaled_to_n():
+    """The hash is the SplitMix64 step, pinned by its published outputs (state 0: first three
+    outputs; state 1234567: first two); a position is floor(h n / 2^64)."""
+    G = 0x9E3779B97F4A7C15
+    assert O.mix64(0) == 0xE220A8397B1DCDAF
+    assert O.mix64(G) == 0x6E789E6AA1B965F4
+    assert O.mix64(2 * G & (2**64 - 1)) == 0x06C45D188009454F
+    assert O.mix64(1234567) == 6457827717110365317
+    assert O.mix64((1234567 + G) & (2**64 - 1)) == 3203168211198807973
+    # call seed 0, tensor 0: draw r hashes the counter r itself
+    n = 1000
+    pos = O.sample_positions(n, 3, 0, 0)
+    assert pos.tolist() == [(0xE220A8397B1DCDAF * n) >> 64, (O.mix64(1) * n) >> 64,
+                            (O.mix64(2) * n) >> 64]
+    # the tensor index enters in the upper word, the call seed by xor
+    pos = O.sample_positions(77, 2, 5, 3)
+    assert pos.tolist() == [(O.mix64(5 ^ (3 << 32) ^ r) * 77) >> 64 for r in range(2)]
+    assert O.call_seed(2, 7) == O.mix64((2 * G + 7) % 2**64)
+    # consecutive calls must not draw (nearly) the same positions
+    a = set(O.sample_positions(100000, 1000, O.call_seed(5, 0), 0).tolist())
+    b = set(O.sample_positions(100000, 1000, O.call_seed(5, 1), 0).tolist())
+    assert len(a & b) < 50
+
+
+def test_positions_are_uniform_over_the_tensor():
+    n, S = 1000, 200000
+    pos = O.sample_positions(n, S, 12345, 7)
+    assert pos.min() >= 0 and pos.max() < n
+    counts = np.bincount(pos, minlength=n)
+    chi2 = ((counts - S / n) ** 2 / (S / n)).sum()
+    assert 800 < chi2 < 1200                              # 999 degrees of freedom: mean 999, sd 45
+    # n close to 2^31: still inside the range and spread over it
+    big = O.sample_positions((1 << 31) - 5, 10000, 1, 0)
+    assert big.min() >= 0 and big.max() < (1 << 31) - 5
+    assert (big < (1 << 30)).mean() == pytest.approx(0.5, abs=0.03)
+    # other tensors and other calls draw other positions
+    assert O.sample_positions(n, 50, 12345, 8).tolist() != pos[:50].tolist()
+    assert O.sample_positions(n, 50, 12346, 7).tolist() != pos[:50].tolist()
+
+
+def test_compress_sampled_is_the_selection_applied_per_tensor():
+    """One iteration of the paper-literal mode = clip, Eq. 5, then for every tensor the
+    generator's positions fed to the selection; packed output; sent entries masked."""
+    rng = np.random.default_rng(43)
+    numel = [400000, 64, 9000]
+    off = [0, 400384, 400896]
+    L = 410112
+    s, seed, it = 0.99, 7, 3
+    w = O.Worker(off, numel, L, 1, 0.9, 0.0, s)
+    g = np.zeros(L, np.float32)
+    for o, n in zip(off, numel):
+        g[o:o + n] = rng.standard_normal(n).astype(np.float32)
+    r, nnz = O.compress_sampled(w, g.copy(), seed=seed, iteration=it)
+    exp_idx = []
+    for j, (o, n) in enumerate(zip(off, numel)):
+        pos = O.sample_positions(n, O.sample_count(n, 0.01), O.call_seed(seed, it), j)
+        ref, _ = _numpy_from_sample(g[o:o + n], pos, O.topk_count(n, s), s)
+        assert nnz[j] == ref.size
+        exp_idx += (ref + o).tolist()
+    assert r.idx.tolist() == exp_idx
+    assert r.val.tobytes() == g[exp_idx].tobytes()
+    assert not w.u[r.idx].any() and not w.v[r.idx].any()
+    k = O.topk_count(400000, s)
+    assert 0.5 * k < nnz[0] < 1.6 * k                     # 40 of 4000 sampled lie above thr
+
+
+def test_sampled_selection_outcomes_fewer_more_exact():
     """n = 100000 at 99.9 %: 1000 sampled elements, k_s = 1, so thr is the sample maximum and
-    the number of entries above it is roughly exponential with mean k: more than 2k pass in
-    about one call in seven, and then exactly the top k must be sent."""
+    the number of entries above it is roughly geometric with mean k: all three outcomes
+    (fewer than k, between k and 2k, precise top-k) occur over 60 calls."""
     rng = np.random.default_rng(53)
     n, s = 100000, 0.999
     k = O.topk_count(n, s)
-    assert O.sample_groups(n, s) == 250
     g = rng.standard_normal(n).astype(np.float32)
     top = _numpy_topk(g, k)
     kinds = set()
@@ -539,16 +660,3 @@ def test_sampled_selection_far_more_than_expected_gives_exact_topk():
             assert r.idx.tolist() == top.tolist()
         kinds.add("exact" if c == k else ("fewer" if c < k else "more"))
     assert kinds == {"exact", "fewer", "more"}
-
-
-def test_sampled_selection_depends_on_seed_and_iteration_only_through_the_sample():
-    rng = np.random.default_rng(47)
-    n, s = 200000, 0.999
-    g = rng.standard_t(3, n).astype(np.float32)
-    outs = []
-    for seed, it in ((1, 0), (1, 0), (1, 1), (2, 0)):
-        w = O.Worker([0], [n], n, 1, 0.0, 0.0, s)
-        r, nnz = O.compress_sampled(w, g.copy(), seed=seed, iteration=it)
-        outs.append(r.idx.tolist())
-    assert outs[0] == outs[1]                          # deterministic
-    assert outs[0] != outs[2] or outs[0] != outs[3]    # another sample, another threshold
