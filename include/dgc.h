@@ -90,7 +90,8 @@ typedef struct dgc_status {
 
 /* Algorithm 4, line "U^k <- 0, V^k <- 0": allocates and zeroes u and v (device
  * memory of cfg->device, arena-sized), the selection scratch and the plan
- * tables.  Synchronous.  The state is owned by the caller until
+ * tables.  Synchronous.  The caller's current device is the same after the
+ * call as before it.  The state is owned by the caller until
  * dgc_state_destroy.  Errors: DGC_EINVAL (NULL, num_tensors < 1, numel < 1,
  * sparsity outside [0,1), sample_ratio outside [0, 0.5], padded arena >=
  * 2^31 elements), DGC_ENOMEM, DGC_ECUDA. */
@@ -102,8 +103,11 @@ int32_t dgc_state_destroy(dgc_state* st);
 /* Sec. 3.3 "Warm-up Training" / Sec. 4.1: change the sparsity between two
  * iterations.  Recomputes k_j = ceil(n_j (1 - s)) (integer arithmetic, parts
  * per 1e9, at least 1), the output offsets and the sampling plan, and uploads
- * them; may reallocate selection scratch (then it synchronises the device).
- * Must not be called while a dgc_compress on this state is still running. */
+ * them; may reallocate selection scratch.  Always synchronises the whole
+ * device, before touching the state and again before returning, so work of
+ * this state that is still running on any stream is waited for.  If the upload
+ * fails (DGC_ENOMEM, DGC_ECUDA) the state is no longer usable: every later
+ * call on it returns DGC_ESTATE until it is destroyed. */
 int32_t dgc_set_sparsity(dgc_state* st, double sparsity);
 
 /* Sec. 4.1: sparsity of warm-up stage 0..4 = 0.75, 0.9375, 0.984375, 0.996,
@@ -185,14 +189,27 @@ int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_id
  *   dense_out             device, dense_len floats, overwritten
  *   workspace             device scratch of at least
  *                         dgc_decode_workspace_bytes(num_workers, dense_len) bytes
- * Precondition (not checked): each list's indices are strictly ascending and
- * inside [0, dense_len) -- what dgc_compress produces.  1 <= num_workers <=
- * DGC_MAX_DECODE_WORKERS.  Asynchronous on `stream`. */
+ * Precondition: each list's indices are strictly ascending and inside
+ * [0, dense_len) -- what dgc_compress produces.  A list that breaks it (a slot
+ * never written, a damaged wire stream) cannot make the call write outside
+ * dense_out or the workspace or read outside the lists: pairs that do not
+ * belong where the order puts them are skipped, the sums of the affected
+ * entries are then unspecified, and dgc_decode_rejected reports how many pairs
+ * were at fault.  1 <= num_workers <= DGC_MAX_DECODE_WORKERS.  Asynchronous on
+ * `stream`. */
 int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lists,
                               const float* const* val_lists, const int64_t* nnz, float* dense_out,
                               int64_t dense_len, void* workspace, int64_t workspace_bytes,
                               void* stream);
 int64_t dgc_decode_workspace_bytes(int32_t num_workers, int64_t dense_len);
+
+/* Input check of the last decode call (any of the dgc_decode_* entry points) that used
+ * `workspace` with these num_workers and dense_len: synchronises `stream` and stores in
+ * *rejected_out the number of pairs whose index was outside [0, dense_len) or not above its
+ * predecessor in the list.  0 = the precondition held.  workspace = NULL asks about the
+ * built-in scratch of dgc_decode_accumulate_static on the current device. */
+int32_t dgc_decode_rejected(int32_t num_workers, int64_t dense_len, const void* workspace,
+                            void* stream, int64_t* rejected_out);
 
 /* The paper has no counterpart to this call: it is dgc_decode_accumulate for callers that
  * must not allocate device memory.  Two kinds of caller are meant.  One runs inside a
@@ -203,11 +220,12 @@ int64_t dgc_decode_workspace_bytes(int32_t num_workers, int64_t dense_len);
  * inputs and the output buffer, but no workspace: the tile-boundary scratch is a fixed
  * DGC_STATIC_DECODE_WORDS * 4 byte (1 MiB) array built into the library, which every GPU that
  * loads the library carries until the process exits.  The call itself performs no cudaMalloc,
- * cudaFree or other allocating call.
+ * cudaFree or other allocating call (the first call on a device looks the array up, which
+ * may make the driver load the library's device code; later calls only launch kernels).
  *   Same arguments, result and preconditions as dgc_decode_accumulate (dense_out is bit for
- * bit the same), minus `workspace`.  Limit: num_workers * (ceil(dense_len / 4096) + 1) must
- * not exceed DGC_STATIC_DECODE_WORDS (e.g. 8 workers up to 134 M dense elements); a larger
- * problem returns DGC_ECAPACITY and enqueues nothing.
+ * bit the same), minus `workspace`.  Limit: num_workers * (ceil(dense_len / 4096) + 1025)
+ * must not exceed DGC_STATIC_DECODE_WORDS (e.g. 8 workers up to 130 M dense elements); a
+ * larger problem returns DGC_ECAPACITY and enqueues nothing.
  *   The first call on each device looks up the array's device address (the device that is
  * current at that call must be the one that owns the buffers); make that first call before
  * starting any stream capture.  All calls on a device share the one array: it still holds the
@@ -226,7 +244,10 @@ int32_t dgc_apply_sgd(float* w, const float* dense_grad, int64_t len, float lr, 
 /* Eq. 5, third term, applied directly: w <- w - lr * sum_k sparse(v_k) without forming
  * the dense gradient.  Only the entries of w that some worker lists change; the result is
  * bit for bit that of dgc_decode_accumulate followed by dgc_apply_sgd (the listed values are
- * summed in worker order from +0, then w[i] <- w[i] - lr * G[i]; elsewhere w - lr * (+0) = w).
+ * summed in worker order from +0, then w[i] <- w[i] - lr * G[i]; elsewhere w - lr * (+0) = w)
+ * for every finite lr >= 0; with lr infinite or NaN the dense form turns every weight into
+ * NaN and this one only the listed ones, and with lr < 0 the dense form turns a weight of -0
+ * into +0 where this one leaves it.
  * Arguments as for dgc_decode_accumulate, with the weight array (device, len floats, read
  * and written) in place of dense_out and the same workspace size.  Asynchronous. */
 int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_lists,
@@ -234,16 +255,17 @@ int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_list
                              int64_t len, float lr, void* workspace, int64_t workspace_bytes,
                              void* stream);
 
-/* Sec. 3.1, encode(): "packs the 32-bit nonzero gradient values and 16-bit run lengths of
- * zeros" -- the wire format behind the compression ratios of Tables 3 and 4.  Entry t is
+/* Sec. 3.1, encode(): 32-bit values of the entries sent plus 16-bit lengths of the zero runs
+ * between them -- the wire format behind the compression ratios of Tables 3 and 4.  Entry t is
  * (runs_out[t], values_out[t]): skip runs_out[t] zeros, then store values_out[t].  More
  * than 65535 zeros in a row are bridged by filler entries (65535, +0.0f), each standing for
  * 65535 zeros and one explicit zero (the paper gives no rule for that case).  Zeros after
  * the last entry are not encoded.  Encoded size = 6 bytes per entry.
  *   idx, val      device, nnz pairs, idx strictly ascending (what dgc_compress emits)
  *   runs_out      device, capacity uint16;  values_out  device, capacity floats
- *   capacity      >= dgc_runlength_max_entries(nnz, dense_len) always suffices; entries
- *                 beyond capacity are dropped (never written) and still counted
+ *   capacity      >= dgc_runlength_max_entries(nnz, dense_len) always suffices; below nnz
+ *                 the call returns DGC_ECAPACITY and enqueues nothing; between the two,
+ *                 entries beyond capacity are dropped (never written) and still counted
  *   count_out     device int64: entries the encoding has (fillers included)
  *   workspace     device, >= dgc_runlength_workspace_bytes(nnz) bytes, 8-byte aligned
  * Asynchronous on `stream`. */
@@ -277,12 +299,13 @@ int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out);
 
 /* Entries the last dgc_compress wrote, in total and per tensor (host outputs, either may be
  * NULL).  select_mode 0: the fixed k_j, no synchronisation.  select_mode 1 (Sec. 5 taken
- * literally): synchronises `stream` and reads the counts.  In that mode the threshold of
- * tensor j is the k_s-th largest |v| of its sample (k_s = ceil(S (1 - s)), S sampled
- * elements: one group of 4 per stratum at a hashed position; tensors of <= 8192 elements are
- * their own sample and use their (k_j + 1)-th largest |v|); every entry with |v| > thr is
- * sent, unless more than 2 k_j pass ("far more than expected"), in which case the exact
- * top-k_j is sent.  The tensors' lists are packed back to back in tensor order (ascending
+ * literally): synchronises `stream` and reads the counts.  In that mode every tensor j is
+ * sampled: S = ceil(sample_ratio n_j) independent uniform draws (draw r at
+ * floor(h n_j / 2^64), h = SplitMix64 step of (call seed xor (j << 32) xor r), call seed =
+ * the same step of (cfg.seed * 0x9E3779B97F4A7C15 + calls completed)); the threshold is the
+ * k_s-th largest sampled |v|, k_s = ceil(S (1 - s)); every entry with |v| > thr is sent,
+ * unless more than 2 k_j pass (the reading of Sec. 5's "far more than expected"), in which
+ * case the exact top-k_j is sent.  The tensors' lists are packed back to back in tensor order (ascending
  * index overall); dgc_max_nnz() is then the capacity bound sum_j min(n_j, 2 k_j), and the
  * out_offset of dgc_layout is not used. */
 int32_t dgc_get_nnz(dgc_state* st, void* stream, int64_t* total_out, int64_t* per_tensor);

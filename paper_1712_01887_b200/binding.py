@@ -67,6 +67,7 @@ _sigs = {
     "dgc_decode_accumulate_static": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
                                                       ctypes.POINTER(_vp), _i64p, _vp,
                                                       ctypes.c_int64, _vp]),
+    "dgc_decode_rejected": (ctypes.c_int32, [ctypes.c_int32, ctypes.c_int64, _vp, _vp, _i64p]),
     "dgc_apply_sgd": (ctypes.c_int32, [_vp, _vp, ctypes.c_int64, ctypes.c_float, _vp]),
     "dgc_decode_accumulate_sgd": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
                                                    ctypes.POINTER(_vp), _i64p, _vp, _vp,
@@ -298,6 +299,17 @@ def decode_accumulate(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[tor
                                       _stream(stream)), "dgc_decode_accumulate")
 
 
+def decode_rejected(num_workers: int, dense_len: int, workspace: Optional[torch.Tensor] = None,
+                    stream=None) -> int:
+    """Pairs the last decode call on `workspace` (None: the built-in scratch of the static
+    variant) skipped or flagged because their index was out of range or out of order."""
+    out = ctypes.c_int64()
+    _check(_lib.dgc_decode_rejected(int(num_workers), int(dense_len),
+                                    None if workspace is None else workspace.data_ptr(),
+                                    _stream(stream), ctypes.byref(out)), "dgc_decode_rejected")
+    return int(out.value)
+
+
 def decode_accumulate_sgd(idx_lists: Sequence[torch.Tensor], val_lists: Sequence[torch.Tensor],
                           dense_out: torch.Tensor, w: torch.Tensor, lr: float,
                           workspace: torch.Tensor, stream=None,
@@ -380,7 +392,7 @@ def decode_accumulate_static(idx_lists: Sequence[torch.Tensor], val_lists: Seque
                              nnz: Optional[Sequence[int]] = None) -> None:
     """dgc_decode_accumulate without a workspace argument, for callers that may not allocate
     device memory: the scratch is a fixed 1 MiB array inside the library.  Raises DgcError
-    (ECAPACITY) when workers x (tiles + 1) exceeds STATIC_DECODE_WORDS.  Calls on one device
+    (ECAPACITY) when workers x (tiles + 1025) exceeds STATIC_DECODE_WORDS.  Calls on one device
     share that scratch, so do not let two of them overlap on the GPU."""
     n = len(idx_lists)
     ip = (_vp * n)(*[_dev(t, torch.int32) for t in idx_lists])

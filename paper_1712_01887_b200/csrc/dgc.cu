@@ -32,6 +32,16 @@ int64_t topk_count(int64_t n, double sparsity) {
   return k;
 }
 
+// Paper-literal mode (Sec. 5): elements drawn from a tensor of n, ceil(ratio * n) in integer
+// arithmetic (parts per 1e9), at least 1, at most n.
+int64_t sample_count(int64_t n, double ratio) {
+  const long long q = std::llround(ratio * 1e9);
+  long long S = ((long long)n * q + 999999999LL) / 1000000000LL;
+  if (S < 1) S = 1;
+  if (S > n) S = n;
+  return S;
+}
+
 // Smallest r with P(Poisson(lambda) >= r) < eps.
 int poisson_rank(double lambda, double eps) {
   if (lambda > 400.0) return (int)std::ceil(lambda + 6.2 * std::sqrt(lambda) + 5.0);
@@ -85,6 +95,7 @@ struct dgc_state {
   int select_smem_keys = 0;
   unsigned long long* d_timeline = nullptr;
   bool alive = false;
+  bool broken = false;   // a sparsity change failed half-way: the plan on the device is not usable
 };
 
 namespace {
@@ -97,6 +108,20 @@ namespace {
       return e__ == cudaErrorMemoryAllocation ? DGC_ENOMEM : DGC_ECUDA; \
     }                                          \
   } while (0)
+
+// Makes `dev` the current device and puts the caller's device back on scope exit.
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { prev = -1; (void)cudaGetLastError(); }
+    if (prev != dev) ok = cudaSetDevice(dev) == cudaSuccess;
+    if (!ok) (void)cudaGetLastError();
+  }
+  ~DeviceGuard() { if (prev >= 0) (void)cudaSetDevice(prev); }
+  DeviceGuard(const DeviceGuard&) = delete;
+  DeviceGuard& operator=(const DeviceGuard&) = delete;
+};
 
 int32_t dev_alloc(dgc_state* st, void** out, size_t bytes) {
   void* ptr = nullptr;
@@ -155,11 +180,21 @@ void build_host_plan(dgc_state* st, double sparsity) {
     const int64_t nseg = (n + kSeg - 1) / kSeg;
     const int64_t nparts = (nseg + kPartSegs - 1) / kPartSegs;
     // sampling plan
-    bool sampled = n > kSmallN;
+    bool sampled = literal || n > kSmallN;
     int groups = 0, rank = 0;
+    int64_t samples = 0;
     double cap_total = (double)n;
     double expect_keys = (double)n;      // keys the select kernel should hold in shared memory
-    if (sampled) {
+    if (literal) {
+      // Sec. 5 as stated: ceil(ratio n) uniform draws from every tensor; thr = the sample's
+      // k_s-th largest key, k_s = ceil(S (1 - s)); about k entries pass, at most 2k are sent,
+      // anything beyond overflows into the exact path
+      samples = sample_count(n, ratio);
+      groups = (int)((samples + 3) / 4);
+      rank = (int)topk_count(samples, sparsity);
+      cap_total = std::min((double)n, 2.0 * (double)k + 1024.0);
+      expect_keys = cap_total;
+    } else if (sampled) {
       const int64_t Q = n / 4;
       int64_t G = (int64_t)std::ceil(ratio * (double)n / 4.0);
       // a sample that holds about 1024 of the entries to send pins the proposal to +-20 %;
@@ -167,8 +202,7 @@ void build_host_plan(dgc_state* st, double sparsity) {
       // cheap (few entries sent) a smaller sample with a wider margin is the better trade:
       // its rank stays within what the sampling kernel's pre-filter handles (one key per thread)
       const double sent = std::max(1.0 - sparsity, 1e-9);
-      // (paper-literal mode keeps the one size rule that its definition states)
-      const double want = literal || sent >= 1.0 / 32.0 ? 1024.0 : sent >= 1.0 / 128.0 ? 256.0 : 128.0;
+      const double want = sent >= 1.0 / 32.0 ? 1024.0 : sent >= 1.0 / 128.0 ? 256.0 : 128.0;
       const int64_t enough = (int64_t)std::ceil(want / sent / 4.0);
       G = std::min<int64_t>(G, enough);
       G = std::max<int64_t>(G, 64);
@@ -177,14 +211,7 @@ void build_host_plan(dgc_state* st, double sparsity) {
       const double lambda = S * (double)k / (double)n;
       rank = poisson_rank(lambda, 1e-9) + 2;
       if (st->cfg.debug_sample_rank > 0) rank = st->cfg.debug_sample_rank;
-      if (literal) {
-        // Sec. 5 as stated: thr = the sample's k_s-th largest key, k_s = ceil(S (1 - s)); about
-        // k entries pass, at most 2k are sent, anything beyond overflows into the exact path
-        rank = (int)topk_count((int64_t)S, sparsity);
-        groups = (int)G;
-        cap_total = std::min((double)n, 2.0 * (double)k + 1024.0);
-        expect_keys = cap_total;
-      } else if (rank >= S / 2) {
+      if (rank >= S / 2) {
         sampled = false;
       } else {
         groups = (int)G;
@@ -195,6 +222,7 @@ void build_host_plan(dgc_state* st, double sparsity) {
     }
     t.rank = sampled ? rank : 0;
     t.groups = sampled ? groups : 0;
+    t.samples = (int32_t)samples;
     if (sampled) {
       t.key_base = (int32_t)st->sample_keys_total;
       t.chunks = (groups + kSampleThreads - 1) / kSampleThreads;
@@ -416,7 +444,8 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   int ndev = 0;
   DGC_CUDA(cudaGetDeviceCount(&ndev));
   if (cfg->device < 0 || cfg->device >= ndev) return DGC_EINVAL;
-  DGC_CUDA(cudaSetDevice(cfg->device));
+  DeviceGuard guard(cfg->device);       // the caller's current device is put back on return
+  if (!guard.ok) return DGC_ECUDA;
   dgc_state* st = new (std::nothrow) dgc_state();
   if (!st) return DGC_ENOMEM;
   st->cfg = *cfg;
@@ -468,7 +497,7 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
 
 int32_t dgc_state_destroy(dgc_state* st) {
   if (!st || !st->alive) return DGC_ESTATE;
-  cudaSetDevice(st->device);
+  DeviceGuard guard(st->device);
   cudaDeviceSynchronize();
   for (void* ptr : st->allocs) cudaFree(ptr);
   st->allocs.clear();
@@ -482,7 +511,12 @@ int32_t dgc_state_destroy(dgc_state* st) {
 int32_t dgc_set_sparsity(dgc_state* st, double sparsity) {
   if (!st || !st->alive) return DGC_ESTATE;
   if (!(sparsity >= 0.0 && sparsity < 1.0)) return DGC_EINVAL;
-  DGC_CUDA(cudaSetDevice(st->device));
+  if (st->broken) return DGC_ESTATE;
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return DGC_ECUDA;
+  // the device is idle before the state is touched: the flush below runs on the default
+  // stream, which does not order itself against non-blocking streams
+  DGC_CUDA(cudaDeviceSynchronize());
   int32_t rc = flush_pending_mask(st, nullptr);   // entries sent by the last call, if deferred
   if (rc != DGC_OK) return rc;
   DGC_CUDA(cudaDeviceSynchronize());
@@ -491,6 +525,7 @@ int32_t dgc_set_sparsity(dgc_state* st, double sparsity) {
   st->plan.sent_bits = st->d_sent_bits;
   st->plan.defer_mask = defer_mask_for(sparsity);
   st->plan.dense_emit = dense_emit_for(sparsity);
+  if (rc != DGC_OK) st->broken = true;            // host plan and device tables no longer agree
   return rc;
 }
 
@@ -533,10 +568,21 @@ static int32_t enqueue_head(dgc_state* st, const float* grad_arena, cudaStream_t
   if (after_norm) DGC_CUDA(cudaEventRecord(after_norm, s));
   if (!st->sample_blocks.empty()) {
     const int grid = (int)st->sample_blocks.size();
-    if (clip && nest) launch(k_sample_threshold<true, true>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
-    else if (clip) launch(k_sample_threshold<true, false>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
-    else if (nest) launch(k_sample_threshold<false, true>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
-    else launch(k_sample_threshold<false, false>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed);
+    const bool lit = st->cfg.select_mode == 1;
+#define DGC_SAMPLE(C, N, L_) \
+    launch(k_sample_threshold<C, N, L_>, grid, kSampleThreads, 0, s, p, grad_arena, m, call_seed)
+    if (lit) {
+      if (clip && nest) DGC_SAMPLE(true, true, true);
+      else if (clip) DGC_SAMPLE(true, false, true);
+      else if (nest) DGC_SAMPLE(false, true, true);
+      else DGC_SAMPLE(false, false, true);
+    } else {
+      if (clip && nest) DGC_SAMPLE(true, true, false);
+      else if (clip) DGC_SAMPLE(true, false, false);
+      else if (nest) DGC_SAMPLE(false, true, false);
+      else DGC_SAMPLE(false, false, false);
+    }
+#undef DGC_SAMPLE
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   return DGC_OK;
@@ -586,7 +632,7 @@ static int32_t enqueue_tail(dgc_state* st, int32_t* out_idx, float* out_val, cud
 
 int32_t dgc_compress(dgc_state* st, const float* grad_arena, int32_t* out_idx, float* out_val,
                      int64_t capacity, void* stream) {
-  if (!st || !st->alive) return DGC_ESTATE;
+  if (!st || !st->alive || st->broken) return DGC_ESTATE;
   if (!grad_arena || !out_idx || !out_val) return DGC_EINVAL;
   if ((reinterpret_cast<uintptr_t>(grad_arena) & 15u) != 0) return DGC_EINVAL;
   if (capacity < st->max_nnz) return DGC_ECAPACITY;
@@ -628,7 +674,7 @@ int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
     return DGC_EINVAL;
   for (int w = 0; w < num_states; ++w) {
     dgc_state* st = states[w];
-    if (!st || !st->alive) return DGC_ESTATE;
+    if (!st || !st->alive || st->broken) return DGC_ESTATE;
     if (st->device != states[0]->device) return DGC_EINVAL;
     if (!grad_arenas[w] || !out_idx[w] || !out_val[w]) return DGC_EINVAL;
     if ((reinterpret_cast<uintptr_t>(grad_arenas[w]) & 15u) != 0) return DGC_EINVAL;
@@ -656,27 +702,35 @@ int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
   // (0.92 ms): a lone pass pays its launch gap and its ramp and drain, concurrent ones hide them.
   DGC_CUDA(cudaEventRecord(r.fork, s));
   for (int i = 0; i < used; ++i) DGC_CUDA(cudaStreamWaitEvent(r.side[i], r.fork, 0));
-  for (int w = 0; w < num_states; ++w) {
+  rc = DGC_OK;
+  for (int w = 0; w < num_states && rc == DGC_OK; ++w) {
     cudaStream_t q = r.side[w % kBatchStreams];
     dgc_state* st = states[w];
-    if ((rc = enqueue_head(st, grad_arenas[w], q, nullptr)) != DGC_OK) return rc;
-    if ((rc = enqueue_stream_pass(st, grad_arenas[w], q)) != DGC_OK) return rc;
-    if ((rc = enqueue_tail(st, out_idx[w], out_val[w], q, nullptr, num_states >= 4)) != DGC_OK) return rc;
+    if ((rc = enqueue_head(st, grad_arenas[w], q, nullptr)) != DGC_OK) break;
+    if ((rc = enqueue_stream_pass(st, grad_arenas[w], q)) != DGC_OK) break;
+    if ((rc = enqueue_tail(st, out_idx[w], out_val[w], q, nullptr, num_states >= 4)) != DGC_OK) break;
     st->iterations += 1;
   }
+  // Join, also after an enqueue error: the side streams were forked from the caller's stream
+  // (inside a capture they belong to it) and what was enqueued on them must be ordered before
+  // whatever the caller does next.
   for (int i = 0; i < used; ++i) {
-    DGC_CUDA(cudaEventRecord(r.join[i], r.side[i]));
-    DGC_CUDA(cudaStreamWaitEvent(s, r.join[i], 0));
+    if (cudaEventRecord(r.join[i], r.side[i]) != cudaSuccess ||
+        cudaStreamWaitEvent(s, r.join[i], 0) != cudaSuccess) {
+      (void)cudaGetLastError();
+      if (rc == DGC_OK) rc = DGC_ECUDA;
+    }
   }
-  return DGC_OK;
+  return rc;
 }
 
 int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_idx_host,
                           float* out_val_host, int64_t capacity, void* stream) {
-  if (!st || !st->alive) return DGC_ESTATE;
+  if (!st || !st->alive || st->broken) return DGC_ESTATE;
   if (!grad_host || !out_idx_host || !out_val_host) return DGC_EINVAL;
   if (capacity < st->max_nnz) return DGC_ECAPACITY;
-  DGC_CUDA(cudaSetDevice(st->device));
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return DGC_ECUDA;
   cudaStream_t s = as_stream(stream);
   int32_t rc;
   void* ptr = nullptr;
@@ -706,27 +760,28 @@ int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_id
   return DGC_OK;
 }
 
-int64_t dgc_decode_workspace_bytes(int32_t num_workers, int64_t dense_len) {
-  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS || dense_len < 0) return DGC_EINVAL;
+}  // extern "C"
+
+// Receive side.  The scratch of a decode call, caller-provided or built in, is
+//   [num_workers x (tiles + 1) tile boundaries][num_workers x kDecodeBoundsBlocks reject counts]
+static int64_t decode_scratch_words(int32_t num_workers, int64_t dense_len) {
   const int64_t tiles = (dense_len + kDecodeTile - 1) / kDecodeTile;
-  return (int64_t)num_workers * (tiles + 1) * 4;
+  return (int64_t)num_workers * (tiles + 1 + kDecodeBoundsBlocks);
 }
 
-int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lists,
-                              const float* const* val_lists, const int64_t* nnz, float* dense_out,
-                              int64_t dense_len, void* workspace, int64_t workspace_bytes,
-                              void* stream) {
-  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
-  if (!idx_lists || !val_lists || !nnz || dense_len < 0 || dense_len >= (int64_t)1 << 31)
-    return DGC_EINVAL;
-  if (dense_len == 0) return DGC_OK;
-  if (!dense_out || !workspace) return DGC_EINVAL;
-  if ((reinterpret_cast<uintptr_t>(dense_out) & 15u) != 0) return DGC_EINVAL;
-  if (workspace_bytes < dgc_decode_workspace_bytes(num_workers, dense_len)) return DGC_ECAPACITY;
+
+// Argument checks and marshalling shared by the decode entry points, then the two launches.
+// `out` is the dense gradient (MODE dense, dense + SGD) or the weights (MODE sparse SGD);
+// `weights` only for dense + SGD.
+template <int MODE>
+static int32_t decode_enqueue(int32_t num_workers, const int32_t* const* idx_lists,
+                              const float* const* val_lists, const int64_t* nnz, float* out,
+                              float* weights, int64_t len, float lr, int32_t* scratch,
+                              cudaStream_t s) {
   DecodeArgs a{};
   int64_t max_nnz = 0;
   for (int w = 0; w < num_workers; ++w) {
-    if (nnz[w] < 0 || nnz[w] > dense_len) return DGC_EINVAL;
+    if (nnz[w] < 0 || nnz[w] > len) return DGC_EINVAL;
     if (nnz[w] > 0 && (!idx_lists[w] || !val_lists[w])) return DGC_EINVAL;
     a.idx[w] = idx_lists[w];
     a.val[w] = val_lists[w];
@@ -734,79 +789,72 @@ int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lis
     max_nnz = std::max(max_nnz, nnz[w]);
   }
   a.num_workers = num_workers;
-  a.num_tiles = (int32_t)((dense_len + kDecodeTile - 1) / kDecodeTile);
-  cudaStream_t s = as_stream(stream);
+  a.num_tiles = (int32_t)((len + kDecodeTile - 1) / kDecodeTile);
+  int32_t* rejected = scratch + (size_t)num_workers * (a.num_tiles + 1);
   int32_t rc;
-  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
-  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
+  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, kDecodeBoundsBlocks);
+  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, scratch, rejected, (long long)len);
   if ((rc = check_launch()) != DGC_OK) return rc;
-  launch(k_decode_tiles<kDecodeDense>, a.num_tiles, kDecodeThreads, 0, s, a,
-         (const int32_t*)workspace, dense_out, (float*)nullptr, dense_len, 0.0f);
+  launch(k_decode_tiles<MODE>, a.num_tiles, kDecodeThreads, 0, s, a, (const int32_t*)scratch, out,
+         weights, (long long)len, lr);
   return check_launch();
+}
+
+static int32_t decode_check_common(int32_t num_workers, const int32_t* const* idx_lists,
+                                   const float* const* val_lists, const int64_t* nnz,
+                                   int64_t len) {
+  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
+  if (!idx_lists || !val_lists || !nnz || len < 0 || len >= (int64_t)1 << 31) return DGC_EINVAL;
+  return DGC_OK;
+}
+
+extern "C" {
+
+int64_t dgc_decode_workspace_bytes(int32_t num_workers, int64_t dense_len) {
+  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS || dense_len < 0) return DGC_EINVAL;
+  return decode_scratch_words(num_workers, dense_len) * 4;
+}
+
+int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lists,
+                              const float* const* val_lists, const int64_t* nnz, float* dense_out,
+                              int64_t dense_len, void* workspace, int64_t workspace_bytes,
+                              void* stream) {
+  int32_t rc = decode_check_common(num_workers, idx_lists, val_lists, nnz, dense_len);
+  if (rc != DGC_OK) return rc;
+  if (dense_len == 0) return DGC_OK;
+  if (!dense_out || !workspace) return DGC_EINVAL;
+  if ((reinterpret_cast<uintptr_t>(dense_out) & 15u) != 0) return DGC_EINVAL;
+  if (workspace_bytes < dgc_decode_workspace_bytes(num_workers, dense_len)) return DGC_ECAPACITY;
+  return decode_enqueue<kDecodeDense>(num_workers, idx_lists, val_lists, nnz, dense_out, nullptr,
+                                      dense_len, 0.0f, (int32_t*)workspace, as_stream(stream));
 }
 
 int32_t dgc_decode_apply_sgd(int32_t num_workers, const int32_t* const* idx_lists,
                              const float* const* val_lists, const int64_t* nnz, float* w,
                              int64_t len, float lr, void* workspace, int64_t workspace_bytes,
                              void* stream) {
-  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
-  if (!idx_lists || !val_lists || !nnz || len < 0 || len >= (int64_t)1 << 31) return DGC_EINVAL;
+  int32_t rc = decode_check_common(num_workers, idx_lists, val_lists, nnz, len);
+  if (rc != DGC_OK) return rc;
   if (len == 0) return DGC_OK;
   if (!w || !workspace) return DGC_EINVAL;
   if (workspace_bytes < dgc_decode_workspace_bytes(num_workers, len)) return DGC_ECAPACITY;
-  DecodeArgs a{};
-  int64_t max_nnz = 0;
-  for (int k = 0; k < num_workers; ++k) {
-    if (nnz[k] < 0 || nnz[k] > len) return DGC_EINVAL;
-    if (nnz[k] > 0 && (!idx_lists[k] || !val_lists[k])) return DGC_EINVAL;
-    a.idx[k] = idx_lists[k];
-    a.val[k] = val_lists[k];
-    a.nnz[k] = (int32_t)nnz[k];
-    max_nnz = std::max(max_nnz, nnz[k]);
-  }
-  a.num_workers = num_workers;
-  a.num_tiles = (int32_t)((len + kDecodeTile - 1) / kDecodeTile);
-  cudaStream_t s = as_stream(stream);
-  int32_t rc;
-  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
-  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
-  if ((rc = check_launch()) != DGC_OK) return rc;
-  launch(k_decode_tiles<kDecodeSparseSgd>, a.num_tiles, kDecodeThreads, 0, s, a,
-         (const int32_t*)workspace, w, (float*)nullptr, len, lr);
-  return check_launch();
+  return decode_enqueue<kDecodeSparseSgd>(num_workers, idx_lists, val_lists, nnz, w, nullptr, len,
+                                          lr, (int32_t*)workspace, as_stream(stream));
 }
 
 int32_t dgc_decode_accumulate_sgd(int32_t num_workers, const int32_t* const* idx_lists,
                                   const float* const* val_lists, const int64_t* nnz,
                                   float* dense_out, float* w, int64_t len, float lr,
                                   void* workspace, int64_t workspace_bytes, void* stream) {
-  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
-  if (!idx_lists || !val_lists || !nnz || len < 0 || len >= (int64_t)1 << 31) return DGC_EINVAL;
+  int32_t rc = decode_check_common(num_workers, idx_lists, val_lists, nnz, len);
+  if (rc != DGC_OK) return rc;
   if (len == 0) return DGC_OK;
   if (!w || !dense_out || !workspace) return DGC_EINVAL;
   if (((reinterpret_cast<uintptr_t>(w) | reinterpret_cast<uintptr_t>(dense_out)) & 15u) != 0)
     return DGC_EINVAL;
   if (workspace_bytes < dgc_decode_workspace_bytes(num_workers, len)) return DGC_ECAPACITY;
-  DecodeArgs a{};
-  int64_t max_nnz = 0;
-  for (int k = 0; k < num_workers; ++k) {
-    if (nnz[k] < 0 || nnz[k] > len) return DGC_EINVAL;
-    if (nnz[k] > 0 && (!idx_lists[k] || !val_lists[k])) return DGC_EINVAL;
-    a.idx[k] = idx_lists[k];
-    a.val[k] = val_lists[k];
-    a.nnz[k] = (int32_t)nnz[k];
-    max_nnz = std::max(max_nnz, nnz[k]);
-  }
-  a.num_workers = num_workers;
-  a.num_tiles = (int32_t)((len + kDecodeTile - 1) / kDecodeTile);
-  cudaStream_t s = as_stream(stream);
-  int32_t rc;
-  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
-  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, (int32_t*)workspace);
-  if ((rc = check_launch()) != DGC_OK) return rc;
-  launch(k_decode_tiles<kDecodeDenseSgd>, a.num_tiles, kDecodeThreads, 0, s, a,
-         (const int32_t*)workspace, dense_out, w, len, lr);
-  return check_launch();
+  return decode_enqueue<kDecodeDenseSgd>(num_workers, idx_lists, val_lists, nnz, dense_out, w,
+                                         len, lr, (int32_t*)workspace, as_stream(stream));
 }
 
 int64_t dgc_runlength_max_entries(int64_t nnz, int64_t dense_len) {
@@ -923,7 +971,8 @@ static int32_t timeline_reset(dgc_state* st) {
 
 int32_t dgc_timeline_enable(dgc_state* st, int32_t on) {
   if (!st || !st->alive) return DGC_ESTATE;
-  DGC_CUDA(cudaSetDevice(st->device));
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return DGC_ECUDA;
   DGC_CUDA(cudaDeviceSynchronize());
   if (on && !st->d_timeline) {
     void* ptr = nullptr;
@@ -947,7 +996,8 @@ int32_t dgc_timeline_read(dgc_state* st, void* stream, uint64_t* ns_out) {
 int32_t dgc_profile_enable(dgc_state* st, int32_t max_calls) {
   if (!st || !st->alive) return DGC_ESTATE;
   if (max_calls < 0) return DGC_EINVAL;
-  DGC_CUDA(cudaSetDevice(st->device));
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return DGC_ECUDA;
   while ((int)st->prof_ev.size() < 6 * max_calls) {
     cudaEvent_t e;
     DGC_CUDA(cudaEventCreate(&e));
@@ -978,7 +1028,11 @@ int32_t dgc_get_nnz(dgc_state* st, void* stream, int64_t* total_out, int64_t* pe
   std::vector<int32_t> h(T);
   if (st->cfg.select_mode == 1) {
     DGC_CUDA(cudaStreamSynchronize(as_stream(stream)));
-    if (st->iterations == 0) std::fill(h.begin(), h.end(), 0);
+    // the device's count of completed calls decides (graph replays do not pass through the host)
+    long long done = 0;
+    DGC_CUDA(cudaMemcpy(&done, st->plan.iter, 8, cudaMemcpyDeviceToHost));
+    st->iterations = done;
+    if (done == 0) std::fill(h.begin(), h.end(), 0);
     else DGC_CUDA(cudaMemcpy(h.data(), st->plan.t_nnz, T * 4, cudaMemcpyDeviceToHost));
   } else {
     for (size_t j = 0; j < T; ++j) h[j] = st->tm[j].k;
@@ -1044,51 +1098,68 @@ constexpr int kMaxDevices = 64;
 std::atomic<int32_t*> g_static_bounds_ptr[kMaxDevices];   // device address per ordinal, 0 = not asked yet
 }  // namespace
 
+// Device address of the built-in scratch on the current device (looked up once per device).
+static int32_t static_decode_scratch(int32_t** out) {
+  int dev = -1;
+  DGC_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return DGC_EINVAL;
+  int32_t* ptr = g_static_bounds_ptr[dev].load(std::memory_order_acquire);
+  if (!ptr) {
+    void* sym = nullptr;
+    DGC_CUDA(cudaGetSymbolAddress(&sym, g_static_decode_bounds));
+    if (!sym) return DGC_ECUDA;
+    ptr = static_cast<int32_t*>(sym);
+    g_static_bounds_ptr[dev].store(ptr, std::memory_order_release);
+  }
+  *out = ptr;
+  return DGC_OK;
+}
+
 extern "C" int32_t dgc_decode_accumulate_static(int32_t num_workers,
                                                  const int32_t* const* idx_lists,
                                                  const float* const* val_lists, const int64_t* nnz,
                                                  float* dense_out, int64_t dense_len, void* stream) {
-  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS) return DGC_EINVAL;
-  if (!idx_lists || !val_lists || !nnz || dense_len < 0 || dense_len >= (int64_t)1 << 31)
-    return DGC_EINVAL;
+  int32_t rc = decode_check_common(num_workers, idx_lists, val_lists, nnz, dense_len);
+  if (rc != DGC_OK) return rc;
   if (dense_len == 0) return DGC_OK;
   if (!dense_out) return DGC_EINVAL;
   if ((reinterpret_cast<uintptr_t>(dense_out) & 15u) != 0) return DGC_EINVAL;
-  const int64_t tiles = (dense_len + kDecodeTile - 1) / kDecodeTile;
-  // the fixed scratch bounds the problem: workers x (tiles + 1) boundary words must fit
-  if ((int64_t)num_workers * (tiles + 1) > (int64_t)DGC_STATIC_DECODE_WORDS) return DGC_ECAPACITY;
-  DecodeArgs a{};
-  int64_t max_nnz = 0;
-  for (int w = 0; w < num_workers; ++w) {
-    if (nnz[w] < 0 || nnz[w] > dense_len) return DGC_EINVAL;
-    if (nnz[w] > 0 && (!idx_lists[w] || !val_lists[w])) return DGC_EINVAL;
-    a.idx[w] = idx_lists[w];
-    a.val[w] = val_lists[w];
-    a.nnz[w] = (int32_t)nnz[w];
-    max_nnz = std::max(max_nnz, nnz[w]);
-  }
-  a.num_workers = num_workers;
-  a.num_tiles = (int32_t)tiles;
+  // the fixed scratch bounds the problem: the boundary and reject words of all workers must fit
+  if (decode_scratch_words(num_workers, dense_len) > (int64_t)DGC_STATIC_DECODE_WORDS)
+    return DGC_ECAPACITY;
   // set-up, once per device, with that device current: the symbol's device address
-  int dev = -1;
-  DGC_CUDA(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= kMaxDevices) return DGC_EINVAL;
-  int32_t* bounds = g_static_bounds_ptr[dev].load(std::memory_order_acquire);
-  if (!bounds) {
-    void* sym = nullptr;
-    DGC_CUDA(cudaGetSymbolAddress(&sym, g_static_decode_bounds));
-    if (!sym) return DGC_ECUDA;
-    bounds = static_cast<int32_t*>(sym);
-    g_static_bounds_ptr[dev].store(bounds, std::memory_order_release);
+  int32_t* scratch = nullptr;
+  if ((rc = static_decode_scratch(&scratch)) != DGC_OK) return rc;
+  // nothing needs clearing: k_decode_bounds writes every boundary word [0, tiles] and every
+  // reject word of every worker before anything reads them, so the previous call's contents
+  // are never seen
+  return decode_enqueue<kDecodeDense>(num_workers, idx_lists, val_lists, nnz, dense_out, nullptr,
+                                      dense_len, 0.0f, scratch, as_stream(stream));
+}
+
+extern "C" int32_t dgc_decode_rejected(int32_t num_workers, int64_t dense_len,
+                                        const void* workspace, void* stream,
+                                        int64_t* rejected_out) {
+  if (num_workers < 1 || num_workers > DGC_MAX_DECODE_WORKERS || dense_len < 0 || !rejected_out)
+    return DGC_EINVAL;
+  *rejected_out = 0;
+  if (dense_len == 0) return DGC_OK;
+  const int32_t* scratch = static_cast<const int32_t*>(workspace);
+  if (!scratch) {
+    if (decode_scratch_words(num_workers, dense_len) > (int64_t)DGC_STATIC_DECODE_WORDS)
+      return DGC_ECAPACITY;
+    int32_t* ptr = nullptr;
+    const int32_t rc = static_decode_scratch(&ptr);
+    if (rc != DGC_OK) return rc;
+    scratch = ptr;
   }
-  // nothing needs clearing: k_decode_bounds writes every boundary word [0, tiles] of every worker
-  // before k_decode_tiles reads it, so the previous call's contents are never seen
-  cudaStream_t s = as_stream(stream);
-  int32_t rc;
-  const int gx = (int)std::min<int64_t>((max_nnz + 1 + 255) / 256, 1024);
-  launch(k_decode_bounds, dim3(gx, num_workers), 256, 0, s, a, bounds);
-  if ((rc = check_launch()) != DGC_OK) return rc;
-  launch(k_decode_tiles<kDecodeDense>, a.num_tiles, kDecodeThreads, 0, s, a, bounds, dense_out,
-         (float*)nullptr, dense_len, 0.0f);
-  return check_launch();
+  const int64_t tiles = (dense_len + kDecodeTile - 1) / kDecodeTile;
+  std::vector<int32_t> h((size_t)num_workers * kDecodeBoundsBlocks);
+  DGC_CUDA(cudaStreamSynchronize(as_stream(stream)));
+  DGC_CUDA(cudaMemcpy(h.data(), scratch + (size_t)num_workers * (tiles + 1), h.size() * 4,
+                      cudaMemcpyDeviceToHost));
+  int64_t total = 0;
+  for (int32_t c : h) total += c;
+  *rejected_out = total;
+  return DGC_OK;
 }

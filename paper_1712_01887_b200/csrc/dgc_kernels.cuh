@@ -45,6 +45,8 @@ constexpr int kPartSegs = 512;         // segments per part (256 Ki elements)
 constexpr int kSmallN = 8192;          // tensors up to this size are not sampled
 constexpr int kMaxSampleGroups = 16384; // float4 groups sampled per tensor at most
 constexpr int kSampleThreads = 512;    // one sampled float4 group per thread and block
+static_assert(kMaxSampleGroups <= 32 * kSampleThreads,
+              "exact mode: at most 32 sampling blocks per tensor, one warp scans their counts");
 constexpr int kSampleSurvivors = 4096;
 constexpr int kSelectThreads = 1024;
 constexpr int kSelectBatchThreads = 512;   // k_select in a batch of several workers
@@ -65,7 +67,6 @@ constexpr int kBigLastBins = 512;
 constexpr int kBigLastStride = 516;    // 513 suffix sums, padded to a multiple of 4 words
 constexpr int kBigStateWords = 64;
 constexpr int kBigNear = 64;           // round-0 digits this close above the proposal's get private bins
-constexpr int kTakeAllTies = 0x3FFFFFFF;   // tie quota meaning "every entry tied with the threshold"
 constexpr int kDecodeTile = 4096;
 constexpr int kDecodeThreads = 256;
 
@@ -77,6 +78,8 @@ struct __align__(16) TensorMeta {   // one per tensor, read-only for the kernels
   int32_t rank, groups;             // sampling: rank of the proposal, float4 groups sampled
   int32_t key_base, chunks;         // sampling: first key in the sample buffer, blocks that sample
   int32_t big, big_slot;            // big: selected by the multi-block path; slot in its tables
+  int32_t samples;                  // paper-literal mode: elements drawn (4 per group, the last
+  int32_t pad_[3];                  // group may be short); otherwise unused
 };
 struct SampleBlock { int32_t tensor, chunk; };   // work item of one k_sample_threshold block
 struct __align__(16) PartMeta {     // one per part (up to kPartSegs segments of one tensor)
@@ -415,12 +418,17 @@ k_sumsq(Plan p, const float* __restrict__ g, double thr_local, int clip_on) {
 // selects.  r is small against the sample, so that block first bounds the
 // answer from below by the rank-r of the per-thread maxima (at least r keys
 // reach it), keeps the few keys that reach the bound and selects among them.
-template <bool CLIP, bool NEST>
+// LITERAL (Sec. 5 taken literally, select_mode 1): the sample is `samples` independent uniform
+// draws of single elements, draw r of tensor j at floor(h n / 2^64), h = mix64(call seed xor
+// (j << 32) xor r); a thread takes draws 4s .. 4s + 3.  Draws beyond `samples` count as key 0,
+// which cannot move the rank-th largest key (rank <= samples).
+template <bool CLIP, bool NEST, bool LITERAL>
 __global__ void __launch_bounds__(kSampleThreads)
 k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_base) {
   pdl_enter();
   timeline_mark(p.timeline, 0);
-  const uint64_t call_seed = seed_base + (uint64_t)__ldcg(p.iter);
+  // hashed, so that consecutive calls draw unrelated positions
+  const uint64_t call_seed = mix64(seed_base + (uint64_t)__ldcg(p.iter));
   __shared__ uint32_t hist[kHistWords(kSampleThreads)];
   __shared__ uint32_t surv[kSampleSurvivors];
   __shared__ int sh[3];
@@ -437,7 +445,36 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   bool have = false;
   {
     const int s = sb.chunk * kSampleThreads + tid;
-    if (s < G) {
+    if (LITERAL && s < G) {
+      const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
+      const uint64_t n = (uint64_t)(uint32_t)(t.end - t.off);
+      uint32_t karr[4] = {0u, 0u, 0u, 0u};
+      uint32_t at[4];
+      float gg[4], uu[4], vv[4];
+      uint32_t sent[4];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const uint32_t r = 4u * (uint32_t)s + (uint32_t)c;
+        const uint64_t h = mix64(call_seed ^ ((uint64_t)(uint32_t)j << 32) ^ (uint64_t)r);
+        // (draws past the sample read position 0 of the tensor and are discarded)
+        at[c] = (uint32_t)t.off + ((int)r < t.samples ? (uint32_t)__umul64hi(h, n) : 0u);
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        gg[c] = __ldg(g + at[c]);
+        uu[c] = __ldcg(p.u + at[c]);
+        vv[c] = __ldcg(p.v + at[c]);
+        sent[c] = p.defer_mask ? __ldcg(p.sent_bits + (at[c] >> 5)) : 0u;
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        if ((sent[c] >> (at[c] & 31u)) & 1u) { uu[c] = 0.0f; vv[c] = 0.0f; }   // pending masking
+        mc_step<CLIP, NEST>(gg[c], coef, m, uu[c], vv[c]);
+        if ((int)(4u * (uint32_t)s + (uint32_t)c) < t.samples) karr[c] = mag_key(vv[c]);
+      }
+      mykeys = make_uint4(karr[0], karr[1], karr[2], karr[3]);
+      have = true;
+    } else if (!LITERAL && s < G) {
       const uint32_t W = (uint32_t)((t.end - t.off) >> 2) / (uint32_t)G;   // groups per stratum
       const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
       // stratum s = groups [s*W, (s+1)*W); position inside it from a hash (multiply-high
@@ -469,7 +506,9 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   // writes them packed into its slice; the last block then selects among a few thousand keys
   // instead of re-reading the whole sample.  (If fewer than `rank` keys of the sample are
   // non-zero the union is short and the answer is 0.)
-  const bool local = t.chunks > 1 && rank <= kSampleThreads;   // (larger ranks: tiny samples)
+  // (larger ranks: tiny samples, or the large samples of the paper-literal mode, which can also
+  // spread over more blocks than the one warp that scans the blocks' counts covers)
+  const bool local = t.chunks > 1 && t.chunks <= 32 && rank <= kSampleThreads;
   if (local) {
     uint32_t* slice = p.sample_keys + t.key_base + sb.chunk * (4 * kSampleThreads);
     const int nv = min(kSampleThreads, G - sb.chunk * kSampleThreads);   // threads with a group
@@ -528,7 +567,6 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   if (local) {
     // the union of the blocks' slices: counts -> offsets (at most 32 blocks per tensor)
     __shared__ int s_off[33];
-    static_assert(kMaxSampleGroups <= 32 * kSampleThreads, "one warp scans the blocks' counts");
     const int first = blockIdx.x - sb.chunk;
     if (tid == 0) s_max = 0u;
     if (tid < 32) {
@@ -879,9 +917,10 @@ k_select(Plan p, int smem_keys) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const TensorMeta t = load_record(p.tm + j);
   const int p0 = t.part_first, pn = t.part_num, k = t.k;
-  const bool tables = pn <= kSelectMaxParts;
   if (j == 0 && tid < 4) p.diag[(parity ^ 1) * 4 + tid] = 0;   // next call's counters
-  if (t.big) return;                                            // k_big_* select this tensor
+  // k_big_* select the big tensors, which include every tensor of more than kSelectMaxParts
+  // parts: the per-part tables below always fit
+  if (t.big || pn > kSelectMaxParts) return;
   if (tid == 0) { s_flag = 0; s_max = 0u; }
   __syncthreads();
   // candidates per part (one load round for all parts), overflow check, compact bases
@@ -909,26 +948,24 @@ k_select(Plan p, int smem_keys) {
         const PartMeta pm = load_record(p.pm + p0 + q);
         c = __ldcg(p.p_count + p0 + q);
         if (c > pm.cap) s_flag = 1;
-        if (tables) s_pcb[q] = pm.cbase;
+        s_pcb[q] = pm.cbase;
       }
       int ex, dummy_e, tot, dummy_t;
       block_excl_scan2(c, 0, sh, ex, dummy_e, tot, dummy_t);
-      if (tables && q < pn) s_pbase[q] = total + ex;
+      if (q < pn) s_pbase[q] = total + ex;
       total += tot;
       __syncthreads();
     }
-    if (tables && tid == 0) s_pbase[pn] = total;
+    if (tid == 0) s_pbase[pn] = total;
     __syncthreads();
   }
   const bool overflow = s_flag != 0;
-  // Paper-literal mode (Sec. 5): what passed the sampled threshold is sent as it is unless it
-  // is "far more than expected" (more than 2k: then the precise top-k); a tensor that is its
-  // own sample (not sampled: every entry is a candidate) sends what exceeds its (k+1)-th key.
+  // Paper-literal mode (Sec. 5): what passed the sampled threshold is sent as it is unless far
+  // more than expected passed (more than 2k: then the precise top-k of the tensor, which all
+  // lie among the candidates).  Every tensor is sampled in that mode.
   const bool literal = p.literal != 0;
-  const bool lit_sampled_all = literal && t.groups > 0 && !overflow && total <= 2 * k;
-  const bool lit_own = literal && t.groups == 0;
-  const bool lit_own_all = lit_own && k + 1 > total;
-  const int rank = lit_own ? k + 1 : k;
+  const bool lit_sampled_all = literal && !overflow && total <= 2 * k;
+  const int rank = k;
   if (!overflow && !literal && total < k && t.groups > 0) {
     const uint32_t tie_key = __ldcg(p.p_thr + p0) - 1u;
     if (tie_fill_parts<THREADS>(p, p0, pn, k, total, t.out_off, tie_key, sh)) {
@@ -959,7 +996,7 @@ k_select(Plan p, int smem_keys) {
     }
     return;
   }
-  const bool in_smem = tables && total <= smem_keys;
+  const bool in_smem = total <= smem_keys;
   const int slices = max(1, (THREADS / 32) / pn);
   uint32_t kmax = 0x7FFFFFFFu;
   uint32_t kbase = 0u;
@@ -989,9 +1026,6 @@ k_select(Plan p, int smem_keys) {
   if (lit_sampled_all) {
     kth = __ldcg(p.p_thr + p0) - 1u;             // every candidate exceeds it (p_thr >= 1 here)
     n_gt = total;
-  } else if (lit_own_all) {
-    kth = 0u;                                    // k = n: everything, zeros included
-    n_gt = 0;
   } else if (in_smem) {
     const int iters = (total + THREADS - 1) / THREADS;
     auto each = [&](auto f) {
@@ -1023,86 +1057,53 @@ k_select(Plan p, int smem_keys) {
         rank, kbase, kmax, hist, sh, n_gt);
   }
   // ties (|v'| == kth) to take, lowest indices first
-  const int quota = lit_sampled_all ? 0 : lit_own_all ? kTakeAllTies : lit_own ? 0 : k - n_gt;
-  const int nnz = lit_sampled_all ? total : lit_own_all ? total : lit_own ? n_gt : k;
+  const int quota = lit_sampled_all ? 0 : k - n_gt;
+  const int nnz = lit_sampled_all ? total : k;
   const int out_off = literal ? 0 : t.out_off;   // paper-literal: k_emit_mask adds the tensor's base
-  if (tables) {
-    // per part: strictly-greater and tied candidates (a single part needs no count: it takes
-    // the whole quota and k_emit_mask stops at the quota by itself)
-    for (int q = tid; q < pn; q += THREADS) { s_gt[q] = 0; s_eq[q] = 0; }
-    __syncthreads();
-    if (pn > 1) {
-      for (int unit = warp; unit < pn * slices; unit += THREADS / 32) {
-        const int q = unit / slices, sl = unit - q * slices;
-        const int b0 = s_pbase[q], c = s_pbase[q + 1] - b0;
-        const float* src = p.cand_val + s_pcb[q];
-        int gt = 0, eq = 0;
-        for (int i = sl * 32 + lane; i < c; i += slices * 32) {
-          const uint32_t key = in_smem ? skeys[b0 + i] : mag_key(__ldcg(src + i));
-          gt += key > kth;
-          eq += key == kth;
-        }
-        gt = __reduce_add_sync(0xFFFFFFFFu, gt);
-        eq = __reduce_add_sync(0xFFFFFFFFu, eq);
-        if (lane == 0) {
-          if (gt) atomicAdd(&s_gt[q], gt);
-          if (eq) atomicAdd(&s_eq[q], eq);
-        }
+  // per part: strictly-greater and tied candidates (a single part needs no count: it takes
+  // the whole quota and k_emit_mask stops at the quota by itself)
+  for (int q = tid; q < pn; q += THREADS) { s_gt[q] = 0; s_eq[q] = 0; }
+  __syncthreads();
+  if (pn > 1) {
+    for (int unit = warp; unit < pn * slices; unit += THREADS / 32) {
+      const int q = unit / slices, sl = unit - q * slices;
+      const int b0 = s_pbase[q], c = s_pbase[q + 1] - b0;
+      const float* src = p.cand_val + s_pcb[q];
+      int gt = 0, eq = 0;
+      for (int i = sl * 32 + lane; i < c; i += slices * 32) {
+        const uint32_t key = in_smem ? skeys[b0 + i] : mag_key(__ldcg(src + i));
+        gt += key > kth;
+        eq += key == kth;
       }
-    } else if (tid == 0) {
-      s_eq[0] = quota;     // upper bound is enough for one part
+      gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+      eq = __reduce_add_sync(0xFFFFFFFFu, eq);
+      if (lane == 0) {
+        if (gt) atomicAdd(&s_gt[q], gt);
+        if (eq) atomicAdd(&s_eq[q], eq);
+      }
     }
-    __syncthreads();
-    if (pn <= 32) {
-      if (warp == 0) {
-        const int gt = lane < pn ? s_gt[lane] : 0, eq = lane < pn ? s_eq[lane] : 0;
-        const int bg = warp_incl_scan(gt) - gt, be = warp_incl_scan(eq) - eq;
-        if (lane < pn) {
-          PartSel ps;
-          ps.kth = kth;
-          ps.quota = max(0, min(quota - be, eq));
-          ps.out_base = out_off + bg + min(be, quota);
-          ps.dense = 0;
-          p.psel[p0 + lane] = ps;
-        }
-      }
-    } else {
-      int run_gt = 0, run_eq = 0;
-      for (int q0 = 0; q0 < pn; q0 += THREADS) {
-        const int q = q0 + tid;
-        const int gt = q < pn ? s_gt[q] : 0, eq = q < pn ? s_eq[q] : 0;
-        int bg, be, tg, te;
-        block_excl_scan2(gt, eq, sh, bg, be, tg, te);
-        bg += run_gt;
-        be += run_eq;
-        if (q < pn) {
-          PartSel ps;
-          ps.kth = kth;
-          ps.quota = max(0, min(quota - be, eq));
-          ps.out_base = out_off + bg + min(be, quota);
-          ps.dense = 0;
-          p.psel[p0 + q] = ps;
-        }
-        run_gt += tg;
-        run_eq += te;
-        __syncthreads();
+  } else if (tid == 0) {
+    s_eq[0] = quota;     // upper bound is enough for one part
+  }
+  __syncthreads();
+  if (pn <= 32) {
+    if (warp == 0) {
+      const int gt = lane < pn ? s_gt[lane] : 0, eq = lane < pn ? s_eq[lane] : 0;
+      const int bg = warp_incl_scan(gt) - gt, be = warp_incl_scan(eq) - eq;
+      if (lane < pn) {
+        PartSel ps;
+        ps.kth = kth;
+        ps.quota = max(0, min(quota - be, eq));
+        ps.out_base = out_off + bg + min(be, quota);
+        ps.dense = 0;
+        p.psel[p0 + lane] = ps;
       }
     }
   } else {
-    // more parts than the tables hold: walk them in chunks, counting from global memory
     int run_gt = 0, run_eq = 0;
     for (int q0 = 0; q0 < pn; q0 += THREADS) {
       const int q = q0 + tid;
-      int gt = 0, eq = 0;
-      if (q < pn) {
-        const int c = __ldcg(p.p_count + p0 + q);
-        const float* src = p.cand_val + __ldg(&p.pm[p0 + q].cbase);
-        for (int i = 0; i < c; ++i) {
-          const uint32_t key = mag_key(__ldcg(src + i));
-          gt += key > kth;
-          eq += key == kth;
-        }
-      }
+      const int gt = q < pn ? s_gt[q] : 0, eq = q < pn ? s_eq[q] : 0;
       int bg, be, tg, te;
       block_excl_scan2(gt, eq, sh, bg, be, tg, te);
       bg += run_gt;
@@ -1976,19 +1977,49 @@ struct DecodeArgs {
   int32_t num_tiles;
 };
 
+// The lists are the caller's: an index outside [0, dense_len) or out of order must neither
+// write outside a bounds row or a tile nor read outside a list.  Tile numbers are clamped to
+// [0, num_tiles] here, k_decode_tiles clamps the boundaries to the list and skips every pair
+// that does not fall into its tile; what was wrong is counted per block (`rejected`:
+// [worker][kDecodeBoundsBlocks], every word rewritten by every call, no atomics, no reset).
+constexpr int kDecodeBoundsBlocks = 1024;   // blocks per worker at most = reject words per worker
+
 __global__ void __launch_bounds__(256)
-k_decode_bounds(const __grid_constant__ DecodeArgs a, int32_t* __restrict__ bounds) {
+k_decode_bounds(const __grid_constant__ DecodeArgs a, int32_t* __restrict__ bounds,
+                int32_t* __restrict__ rejected, long long dense_len) {
   pdl_enter();
   // bounds[w * (num_tiles + 1) + t] = first position in list w whose index >= t * tile
+  __shared__ int s_bad[256 / 32];
   const int w = blockIdx.y;
-  const int n = a.nnz[w];
+  const long long n = a.nnz[w];
   const int32_t* idx = a.idx[w];
   int32_t* b = bounds + (size_t)w * (a.num_tiles + 1);
-  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i <= n; i += gridDim.x * blockDim.x) {
-    const int t_prev = (i == 0) ? -1 : (__ldg(idx + i - 1) / kDecodeTile);
-    const int t_cur = (i == n) ? a.num_tiles : (__ldg(idx + i) / kDecodeTile);
-    for (int t = t_prev + 1; t <= t_cur; ++t) b[t] = i;
+  auto tile_of = [&](int x) { return x < 0 ? 0 : min(x / kDecodeTile, a.num_tiles); };
+  int bad = 0;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i <= n;
+       i += (long long)gridDim.x * blockDim.x) {
+    const int prev = i == 0 ? -1 : __ldg(idx + i - 1);
+    const int cur = i == n ? 0x7FFFFFFF : __ldg(idx + i);
+    // pair i breaks the precondition: outside the dense range, or not above its predecessor
+    if (i < n && ((unsigned long long)(long long)cur >= (unsigned long long)dense_len ||
+                  (i > 0 && cur <= prev)))
+      ++bad;
+    const int t_prev = i == 0 ? -1 : tile_of(prev);
+    const int t_cur = i == n ? a.num_tiles : tile_of(cur);
+    for (int t = t_prev + 1; t <= t_cur; ++t) b[t] = (int32_t)i;
   }
+  bad = __reduce_add_sync(0xFFFFFFFFu, bad);
+  if ((threadIdx.x & 31) == 0) s_bad[threadIdx.x >> 5] = bad;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int tot = 0;
+    for (int q = 0; q < 256 / 32; ++q) tot += s_bad[q];
+    rejected[w * kDecodeBoundsBlocks + blockIdx.x] = tot;
+  }
+  // the words of blocks that this launch does not have
+  if (blockIdx.x == 0)
+    for (int q = gridDim.x + threadIdx.x; q < kDecodeBoundsBlocks; q += blockDim.x)
+      rejected[w * kDecodeBoundsBlocks + q] = 0;
 }
 
 // MODE 0: the tile of the dense gradient is written out (zero-fill fused).
@@ -2021,9 +2052,10 @@ k_decode_tiles(const __grid_constant__ DecodeArgs a, const int32_t* __restrict__
       const int w = w0 + tid;
       int lo = 0, len = 0;
       if (w < N) {
+        // (clamped to the list: a list that is not ascending leaves boundaries unordered)
         const int32_t* b = bounds + (size_t)w * (a.num_tiles + 1);
-        lo = __ldg(b + t);
-        len = __ldg(b + t + 1) - lo;
+        lo = min(max(__ldg(b + t), 0), a.nnz[w]);
+        len = min(max(__ldg(b + t + 1), lo), a.nnz[w]) - lo;
         s_lo[w] = lo;
       }
       const int incl = warp_incl_scan(len);
@@ -2056,8 +2088,10 @@ k_decode_tiles(const __grid_constant__ DecodeArgs a, const int32_t* __restrict__
       }
       myw = lo;
       const int pos = s_lo[lo] + (q - s_cum[lo]);
-      l = __ldg(a.idx[lo] + pos) - (int)base;
+      l = (int)((unsigned)__ldg(a.idx[lo] + pos) - (unsigned)base);
       v = __ldg(a.val[lo] + pos);
+      // a pair that is not of this tile (bad index; k_decode_bounds counted it) is skipped
+      if ((unsigned)l >= (unsigned)kDecodeTile || base + l >= dense_len) myw = -1;
     }
     // workers present in this chunk (block-uniform bounds)
     int wfirst = 0, wlast = N - 1;
@@ -2144,7 +2178,7 @@ k_sgd(float* __restrict__ w, const float* __restrict__ G, long long len, float l
 }
 
 // ------------------------------------------------------------------ wire format: values + 16-bit zero run lengths
-// Sec. 3.1: encode() packs the 32-bit non-zero values and 16-bit run lengths of zeros.
+// Sec. 3.1, encode(): 32-bit values of the sent entries + 16-bit lengths of the zero runs.
 // Entry t = (run_t, value_t): run_t zeros are skipped, then value_t is stored.  A gap of
 // more than 65535 zeros is bridged by filler entries (65535, +0.0f), each standing for 65535
 // zeros and one slot holding an explicit zero (the paper gives no rule; this is the reading).

@@ -37,7 +37,8 @@ def test_host_only_calls(B):
     assert [B.warmup_sparsity(i) for i in range(5)] == [0.75, 0.9375, 0.984375, 0.996, 0.999]
     with pytest.raises(B.DgcError):
         B.warmup_sparsity(5)
-    assert B.decode_workspace_bytes(8, 4096 * 10) == 8 * 11 * 4
+    # per worker: 11 tile boundaries + 1024 input-check words
+    assert B.decode_workspace_bytes(8, 4096 * 10) == 8 * (11 + 1024) * 4
     assert B.decode_workspace_bytes(0, 10) < 0 and B.decode_workspace_bytes(65, 10) < 0
     assert isinstance(B.launch_count(), int)
 

@@ -393,6 +393,78 @@ def test_decode_edge_cases(P):
         P.receive_side(idx, val, L, w0, lr=0.05)
 
 
+def test_decode_skips_and_reports_indices_that_break_the_precondition(P):
+    """A list with an index outside [0, dense_len), a repeated one or one out of order must
+    not make the receive side write outside its output or workspace.  The buffers are
+    allocated with slack beyond the dense_len that is passed, the bad indices point into that
+    slack, so the test cannot fault whatever the kernels do (negative and huge indices take
+    the same guards: tile numbers are clamped, tile offsets compared as unsigned); the slack must stay untouched, the good
+    entries must still be summed, and dgc_decode_rejected must count the bad pairs."""
+    from paper_1712_01887_b200 import binding as B
+    dense_len, slack = 3 * 4096 + 100, 4 * 4096
+    N = 3
+    good = [np.array([5, 4096, 4097, 9000, dense_len - 1], np.int32),
+            np.array([5, 100, 9000], np.int32),
+            np.array([0, 12000], np.int32)]
+    vals = [np.arange(1, a.size + 1, dtype=np.float32) * (w + 1) for w, a in enumerate(good)]
+    ref = np.zeros(dense_len, np.float32)
+    for a, v in zip(good, vals):
+        np.add.at(ref, a, v)
+
+    def run(lists_i, lists_v, fn):
+        di = [torch.from_numpy(a).cuda() for a in lists_i]
+        dv = [torch.from_numpy(v).cuda() for v in lists_v]
+        out = torch.full((dense_len + slack,), 7.0, dtype=torch.float32, device="cuda")
+        ws_bytes = B.decode_workspace_bytes(N, dense_len)
+        ws = torch.full((ws_bytes + 4096,), 0x5A, dtype=torch.uint8, device="cuda")
+        fn(di, dv, out[:dense_len], ws[:ws_bytes])
+        torch.cuda.synchronize()
+        assert bool((out[dense_len:] == 7.0).all()), "wrote past dense_len"
+        assert bool((ws[ws_bytes:] == 0x5A).all()), "wrote past the workspace"
+        return out[:dense_len].cpu().numpy(), B.decode_rejected(N, dense_len, ws[:ws_bytes])
+
+    dense = lambda di, dv, out, ws: B.decode_accumulate(di, dv, out, ws)      # noqa: E731
+    got, rej = run(good, vals, dense)
+    assert got.tobytes() == ref.tobytes() and rej == 0
+    # (a) indices beyond dense_len at the end of a list (ascending, so the rest is intact)
+    bad_i = [np.concatenate([good[0], [dense_len, dense_len + 5000]]).astype(np.int32), good[1],
+             good[2]]
+    bad_v = [np.concatenate([vals[0], [99.0, 98.0]]).astype(np.float32), vals[1], vals[2]]
+    got, rej = run(bad_i, bad_v, dense)
+    assert got.tobytes() == ref.tobytes() and rej == 2
+    # (b) an index listed twice by one worker: reported (which of the two values lands first is
+    #     unspecified, so only the other entries are compared)
+    bad_i = [good[0], np.array([5, 100, 100, 9000], np.int32), good[2]]
+    bad_v = [vals[0], np.array([1.0, 2.0, 2.5, 3.0], np.float32) * 2, vals[2]]
+    got, rej = run(bad_i, bad_v, dense)
+    keep = np.ones(dense_len, bool)
+    keep[100] = False
+    assert got[keep].tobytes() == ref[keep].tobytes() and rej == 1
+    # (c) out of order (an unwritten slot in the middle): no fault, no stray write, reported;
+    #     the sums of the affected list are unspecified, the other workers' entries are intact
+    bad_i = [good[0], good[1], np.array([12000, 0, 7], np.int32)]
+    bad_v = [vals[0], vals[1], np.array([1.0, 2.0, 3.0], np.float32)]
+    got, rej = run(bad_i, bad_v, dense)
+    assert rej >= 1
+    only01 = np.zeros(dense_len, np.float32)
+    for a, v in zip(good[:2], vals[:2]):
+        np.add.at(only01, a, v)
+    untouched = np.ones(dense_len, bool)
+    untouched[[12000, 0, 7]] = False
+    assert got[untouched].tobytes() == only01[untouched].tobytes()
+    # the fused forms take the same guarded path
+    w0 = np.linspace(-1, 1, dense_len + slack).astype(np.float32)
+
+    def sparse_sgd(di, dv, out, ws):
+        out.copy_(torch.from_numpy(w0[:dense_len]).cuda())
+        B.decode_apply_sgd(di, dv, out, 0.5, ws)
+    bad_i = [np.concatenate([good[0], [dense_len + 1]]).astype(np.int32), good[1], good[2]]
+    bad_v = [np.concatenate([vals[0], [99.0]]).astype(np.float32), vals[1], vals[2]]
+    got, rej = run(bad_i, bad_v, sparse_sgd)
+    assert rej == 1
+    assert got.tobytes() == (w0[:dense_len] - np.float32(0.5) * ref).astype(np.float32).tobytes()
+
+
 def test_runlength_wire_format_matches_oracle(P):
     """Sec. 3.1 encode(): values + 16-bit zero run lengths, against the oracle bit for bit;
     then back through decode and the dense sum."""
@@ -539,20 +611,24 @@ def test_deferred_masking_without_reading_state_between_iterations(P, sparsity):
     pair.close()
 
 
-@pytest.mark.parametrize("sparsity,numel,iters", [
-    (0.999, [100000, 8192, 64, 70001, 600000, 1 << 21], 12),
-    (0.99, [1 << 22, 300000, 5000, 9000], 4),           # the 2^22 tensor takes the multi-block path
-    (0.75, [200000, 1000], 3),
+@pytest.mark.parametrize("sparsity,numel,iters,ratio", [
+    (0.999, [100000, 8192, 64, 70001, 600000, 1 << 21, 1, 3], 12, 0.01),
+    (0.99, [1 << 22, 300000, 5000, 9000], 4, 0.01),     # the 2^22 tensor takes the multi-block path
+    (0.75, [200000, 1000], 3, 0.01),
+    (0.999, [(1 << 23) + 5, 70001], 3, 0.01),           # 83,887 draws: more than 32 sampling blocks
+    (0.99, [1 << 23, 513], 2, 0.01),                    # the same with sample rank 839 (> one block)
+    (0.999, [1 << 22, 100000, 2000], 4, 0.001),         # the paper's smallest sample: 0.1 %
 ])
-def test_paper_literal_sampled_selection_matches_oracle(P, sparsity, numel, iters):
-    """select_mode = 1: Sec. 5 as stated (threshold from the sample, variable count).  The
-    oracle draws the same sample (same counter-based hash); indices, values, per-tensor counts
-    and state must agree bit for bit, over several iterations and all three outcomes (fewer
-    than k, more than k, more than 2k -> exact top-k)."""
+def test_paper_literal_sampled_selection_matches_oracle(P, sparsity, numel, iters, ratio):
+    """select_mode = 1: Sec. 5 as stated (ceil(ratio n) uniform draws per tensor, threshold =
+    the sample's ceil(S (1 - s))-th largest |v|, strict compare, exact top-k only when more
+    than 2k pass; variable count).  The oracle takes the positions from the same counter-based
+    generator; indices, values, per-tensor counts and state must agree bit for bit, over
+    several iterations and all outcomes (fewer than k, more than k, more than 2k)."""
     from oracle import dgc_oracle as O
     from paper_1712_01887_b200 import binding as B
     seed = 77
-    st = B.State(numel, 4, 0.9, 1.0, sparsity, seed=seed, select_mode=1)
+    st = B.State(numel, 4, 0.9, 1.0, sparsity, seed=seed, select_mode=1, sample_ratio=ratio)
     L, off = st.arena_len, st.arena_offset
     cpu = O.Worker(off, numel, L, 4, 0.9, 1.0, sparsity)
     assert st.max_nnz == int(np.minimum(np.asarray(numel), 2 * cpu.k).sum())
@@ -568,10 +644,10 @@ def test_paper_literal_sampled_selection_matches_oracle(P, sparsity, numel, iter
         status = st.status()
         total, per = st.nnz()
         snap = (cpu.u.copy(), cpu.v.copy())
-        r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t)
+        r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t, sample_ratio=ratio)
         if np.float32(status.clip_coef).tobytes() != np.float32(r.coef).tobytes():
             cpu.u[:], cpu.v[:] = snap
-            r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t,
+            r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t, sample_ratio=ratio,
                                         coef_override=status.clip_coef)
         assert per.tolist() == nnz.tolist(), (t, per, nnz)
         assert total == r.idx.size
@@ -581,8 +657,8 @@ def test_paper_literal_sampled_selection_matches_oracle(P, sparsity, numel, iter
         assert u.tobytes() == cpu.u.tobytes() and v.tobytes() == cpu.v.tobytes()
         for c, k in zip(nnz, cpu.k):
             kinds.add("k" if c == k else ("fewer" if c < k else "more"))
-    if sparsity == 0.999:
-        assert {"fewer", "more"} <= kinds
+    if sparsity == 0.999 and iters >= 12:
+        assert {"fewer", "more", "k"} <= kinds
     st.close()
 
 

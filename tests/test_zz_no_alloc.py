@@ -39,6 +39,16 @@ def test_static_decode_matches_workspace_decode_twice_in_a_row():
         # same tolerance as the other decode tests: none (bit-exact)
         assert torch.equal(out.view(torch.int32), ref.view(torch.int32))
         assert not torch.isnan(out).any()
+        assert B.decode_rejected(workers, dense_len) == 0     # the built-in scratch's input check
+        # what the entry point is for: once the first call on the device has looked the scratch
+        # up, a call takes no device memory, neither from the driver nor from torch's allocator
+        free0, _ = torch.cuda.mem_get_info()
+        held0, reserved0 = torch.cuda.memory_allocated(), torch.cuda.memory_reserved()
+        B.decode_accumulate_static(idx, val, out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free0
+        assert (torch.cuda.memory_allocated(), torch.cuda.memory_reserved()) == (held0, reserved0)
+        assert torch.equal(out.view(torch.int32), ref.view(torch.int32))
 
 
 def test_static_decode_rejects_problems_beyond_its_fixed_scratch():
@@ -46,7 +56,8 @@ def test_static_decode_rejects_problems_beyond_its_fixed_scratch():
         pytest.fail("no CUDA device: the gpu tests need a B200")
     from paper_1712_01887_b200 import binding as B
     workers = 64
-    tiles_allowed = B.STATIC_DECODE_WORDS // workers - 1          # tiles of 4096 elements
+    # per worker: one boundary word per tile of 4096 elements, one more, and 1024 check words
+    tiles_allowed = B.STATIC_DECODE_WORDS // workers - 1 - 1024
     too_long = (tiles_allowed + 1) * 4096
     empty_i = [torch.zeros(0, dtype=torch.int32, device="cuda") for _ in range(workers)]
     empty_v = [torch.zeros(0, dtype=torch.float32, device="cuda") for _ in range(workers)]
