@@ -41,11 +41,25 @@ from paper_1712_01887_b200 import inputs as I  # noqa: E402
 
 METRIC = "compressed gradient elements/s"
 UNIT = "elements/s"
-POOL = 2            # distinct pre-generated gradients per worker
+E2E_POOL = 2        # pinned host gradients per worker for the end-to-end leg
 LR = 0.01
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_update_emit launch, from the ncu capture
-# summarised in profiles/k_update_emit_resnet50_ncu_full.md (same per-launch size as the bench)
-NCU_TRAFFIC_BYTES = {"resnet50": 307.17e6 + 150.27e6}
+TRAFFIC_JSON = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+
+
+def _pool_size(wl) -> int:
+    """Distinct pre-generated gradients per worker: the workload's stated iteration count (10
+    for the ResNet-50- and LSTM-shaped sets), so that consecutive steps see fresh gradients."""
+    return max(2, min(int(wl.iterations), 10))
+
+
+def _ncu_traffic(workload: str, kernel: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of `kernel` on `workload`,
+    from the committed ncu summaries (profiles/ncu_dram_traffic.json); None if not captured."""
+    try:
+        with open(TRAFFIC_JSON) as f:
+            return float(json.load(f)[workload][kernel]["dram_bytes_per_launch"])
+    except (OSError, KeyError, ValueError, TypeError):
+        return None
 
 
 def _peaks():
@@ -130,49 +144,67 @@ def _layout(wl):
     return I.packed_layout(wl.numel, align=512)
 
 
-def _make_pool(wl, n_workers, rank, pool=POOL):
-    """pool x n_workers host gradients (pinned), generated once, seeded."""
-    import torch
+def _host_gradients(wl, n_workers, rank, pool):
+    """pool x n_workers host gradients (numpy), generated once, seeded; a few host threads
+    fill them side by side (numpy's generators release the interpreter lock)."""
+    from concurrent.futures import ThreadPoolExecutor
     off, L = _layout(wl)
+
+    def one(wi):
+        w, i = wi
+        a = np.zeros(L, np.float32)
+        I.fill(wl, a, off, worker=rank * 1000 + w, iteration=i)
+        return a
+
+    jobs = [(w, i) for w in range(n_workers) for i in range(pool)]
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        flat = list(ex.map(one, jobs))
+    return off, L, [flat[w * pool:(w + 1) * pool] for w in range(n_workers)]
+
+
+def _make_pool(wl, n_workers, rank, pool=E2E_POOL):
+    """pool x n_workers pinned host gradients (for the modes that copy from the host)."""
+    import torch
+    off, L, rows = _host_gradients(wl, n_workers, rank, pool)
     hosts = []
-    for w in range(n_workers):
-        row = []
-        for i in range(pool):
-            t = torch.zeros(L, dtype=torch.float32).pin_memory()
-            I.fill(wl, t.numpy(), off, worker=rank * 1000 + w, iteration=i)
-            row.append(t)
-        hosts.append(row)
+    for row in rows:
+        out = []
+        for a in row:
+            t = torch.empty(L, dtype=torch.float32).pin_memory()
+            t.numpy()[:] = a
+            out.append(t)
+        hosts.append(out)
     return off, L, hosts
 
 
-def run_ours(args):
+def measure(args, wl, rank, world, dev, headline):
+    """All timings of one workload.  `headline`: also the end-to-end leg, the wire format, the
+    timeline and the CPU baseline (the second target workload reports the device timings only)."""
     import torch
     import torch.distributed as dist
-    from paper_1712_01887_b200 import build
-    build.build()
     from paper_1712_01887_b200 import binding as B
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    dev = torch.cuda.current_device()
-    wl = I.workload(args.workload) if args.workload != "sweep" else I.workload("sweep", n=args.n)
-    if args.clip is not None:
-        wl.clip_threshold = args.clip
-    if args.sparsity is not None:
-        wl.sparsity = args.sparsity
     NW = args.workers or wl.num_workers
-    off, L, hosts = _make_pool(wl, NW, rank)
+    POOL = _pool_size(wl)
+    off, L, grads = _host_gradients(wl, NW, rank, POOL)
     total = wl.total
     states = [B.State(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold, wl.sparsity,
                       sample_ratio=wl.sample_ratio, seed=I.BASE_SEED + w, device=dev)
               for w in range(NW)]
     assert states[0].arena_len == L and np.array_equal(states[0].arena_offset, off)
     nnz = states[0].max_nnz
-    pool = [[h.cuda() for h in row] for row in hosts]
+    pool = [[torch.from_numpy(a).cuda() for a in row] for row in grads]
+    hosts = None
+    if headline and not args.no_e2e:
+        hosts = []
+        for row in grads:
+            pinned = []
+            for a in row[:E2E_POOL]:
+                t = torch.empty(L, dtype=torch.float32).pin_memory()
+                t.numpy()[:] = a
+                pinned.append(t)
+            hosts.append(pinned)
+    del grads
     out_i = [torch.empty(nnz, dtype=torch.int32, device="cuda") for _ in range(NW)]
     out_v = [torch.empty(nnz, dtype=torch.float32, device="cuda") for _ in range(NW)]
     dense = torch.empty(L, dtype=torch.float32, device="cuda")
@@ -221,7 +253,7 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    K, W = args.steps, args.warmup
+    K, W, R = args.steps, args.warmup, max(1, args.repeats)
     for t in range(W):
         step(t)
     barrier()
@@ -249,43 +281,51 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    launches0 = B.launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+    flush = None
     if args.flush_l2:
         # cold-cache variant for working sets that fit the 126 MB L2: a 256 MB buffer is
         # rewritten before every step, outside the per-step event pairs that are summed
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
-        pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
-                 for _ in range(K)]
-        for t in range(W, W + K):
-            flush.zero_()
-            pairs[t - W][0].record()
-            step(t)
-            pairs[t - W][1].record()
+    # the timed region, R times: exactly K steps each, bracketed by barrier + synchronize
+    rep_ms, launches = [], 0
+    t_next = W
+    for _ in range(R):
+        launches0 = B.launch_count()
         barrier()
-        ms = sum(a.elapsed_time(b) for a, b in pairs)
-        del flush
-    else:
-        e0.record()
-        for t in range(W, W + K):
-            step(t)
-        e1.record()
-        barrier()
-        ms = e0.elapsed_time(e1)
-    launches = B.launch_count() - launches0
+        if flush is not None:
+            pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                     for _ in range(K)]
+            for q in range(K):
+                flush.zero_()
+                pairs[q][0].record()
+                step(t_next + q)
+                pairs[q][1].record()
+            barrier()
+            ms = sum(a.elapsed_time(b) for a, b in pairs)
+        else:
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for q in range(K):
+                step(t_next + q)
+            e1.record()
+            barrier()
+            ms = e0.elapsed_time(e1)
+        t_next += K
+        launches = B.launch_count() - launches0
+        rep_ms.append(max_over_ranks(ms))
+    del flush
     if graphs is not None:
         launches = graph_launches * K              # kernels inside the replayed graphs
         del graphs
     clocks = sampler.stop() if rank == 0 else None
-    ms = max_over_ranks(ms)
+    ms = float(np.median(rep_ms))
 
     # the same K steps once more with stage events recorded inside every dgc_compress: the
     # dominant kernel's duration for the roofline (the events themselves cost about 3 us per
     # stage, which is why the headline region above runs without them)
     for s in states:
         s.profile_enable(K)
-    for t in range(W + K, W + 2 * K):          # one stream: overlapped kernels cannot be timed
+    for t in range(t_next, t_next + K):        # one stream: overlapped kernels cannot be timed
         for w in range(NW):
             states[w].compress(pool[w][t % POOL], out_i[w], out_v[w])
         receive_side()
@@ -295,7 +335,8 @@ def run_ours(args):
     for s in states:
         s.profile_enable(0)
 
-    # compress-only timing, one stream (same states keep evolving)
+    # compress-only timing, one stream (same states keep evolving): one worker's calls back to
+    # back, the deployment the paper describes (one worker per GPU)
     c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     c0.record()
@@ -328,24 +369,26 @@ def run_ours(args):
                "fused_sparse_decode_sgd_ms": _time(
                    lambda: B.decode_apply_sgd(out_i, out_v, weights, LR, ws))}
 
-    # the paper's wire format (values + 16-bit zero run lengths) of one worker's list
-    runs, _vals = B.encode_runlength(out_i[0], out_v[0], L)
-    enc_ms = _time(lambda: B.encode_runlength(out_i[0], out_v[0], L), reps=5)
-    wire = {"entries": int(runs.numel()), "bytes": int(runs.numel()) * 6,
-            "compression_ratio": total * 4 / max(int(runs.numel()) * 6, 1),
-            "encode_ms_with_count_readback": enc_ms}
+    wire = None
+    if headline:
+        # the paper's wire format (values + 16-bit zero run lengths) of one worker's list
+        runs, _vals = B.encode_runlength(out_i[0], out_v[0], L)
+        enc_ms = _time(lambda: B.encode_runlength(out_i[0], out_v[0], L), reps=5)
+        wire = {"entries": int(runs.numel()), "bytes": int(runs.numel()) * 6,
+                "compression_ratio": total * 4 / max(int(runs.numel()) * 6, 1),
+                "encode_ms_with_count_readback": enc_ms}
 
     # end to end through the host-buffer entry point: H2D of every gradient and D2H of the
     # sparse lists inside the timed region
     e2e = None
-    if not args.no_e2e:
+    if hosts is not None:
         hi = [torch.empty(nnz, dtype=torch.int32).pin_memory() for _ in range(NW)]
         hv = [torch.empty(nnz, dtype=torch.float32).pin_memory() for _ in range(NW)]
         KE = max(1, min(K, args.e2e_steps))
 
         def e2e_step(t):
             for w in range(NW):
-                states[w].compress_host(hosts[w][t % POOL], hi[w], hv[w])
+                states[w].compress_host(hosts[w][t % E2E_POOL], hi[w], hv[w])
             # the lists a receiver would get are on the host now; the receive side runs on the
             # device copies the call also left in the state's output staging
             for w in range(NW):
@@ -365,11 +408,6 @@ def run_ours(args):
                "h2d_bytes_per_step": NW * (L * 4 + nnz * 8), "d2h_bytes_per_step": NW * nnz * 8,
                "ms_per_step": dt / KE * 1e3, "steps": KE}
 
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
     peak, peak_src = _peaks()
     k_ms = float(np.mean(kern_ms))
     alg_bytes = 20.0 * total                       # read g,u,v + write u,v per real element
@@ -379,7 +417,7 @@ def run_ours(args):
     # timeline aid: first and last block start of every kernel), with the GPU kept busy while
     # the host enqueues the step so that the step runs as it does in the timed loop
     timeline = None
-    if args.timeline:
+    if args.timeline and headline and rank == 0:
         for s_ in states:
             s_.timeline_enable(True)
         for t in range(3):
@@ -407,16 +445,18 @@ def run_ours(args):
     recv_bytes = 8.0 * NW * nnz + 4.0 * L + (12.0 if args.separate_receive else 8.0) * L
     step_bytes = NW * compress_bytes + recv_bytes
     step_gbs = step_bytes / (ms / K * 1e-3) / 1e9
-    cpu = None if args.no_cpu_baseline else cpu_baseline(wl, budget_s=args.cpu_seconds)
-    line = {
-        "metric": METRIC, "value": whole_job_value(NW * total, K, world, ms), "unit": UNIT,
-        "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+    for s_ in states:
+        s_.close()
+    res = {
+        "value": whole_job_value(NW * total, K, world, ms), "ms_per_step": ms / K,
+        "repeats": {"n": R, "ms_per_step": [x / K for x in rep_ms],
+                    "min": min(rep_ms) / K, "max": max(rep_ms) / K,
+                    "reported": "median of the repeats, each exactly `steps` steps"},
         "config": {"workload": wl.name, "tensors": len(wl.shapes), "elements": total,
                    "simulated_workers": NW, "sparsity": wl.sparsity, "momentum": wl.momentum,
                    "clip_threshold": wl.clip_threshold, "sample_ratio": wl.sample_ratio,
                    "nnz_per_worker": nnz,
+                   "gradients": f"{POOL} distinct pre-generated gradients per worker, cycled",
                    "compress_call": "dgc_compress per worker on %d streams" % NS if args.no_batch
                    else "dgc_compress_batch (all workers in one call)",
                    "streams": NS,
@@ -439,17 +479,72 @@ def run_ours(args):
                                       "same K steps",
                      "algorithmic_bytes_per_launch": alg_bytes,
                      "traffic": args.traffic if args.traffic is not None
-                     else NCU_TRAFFIC_BYTES.get(wl.name)},
+                     else _ncu_traffic(wl.name, "k_update_emit")},
         "stages_ms": dict(zip(["norm", "sample", "stream", "select", "emit"],
                               [float(x) for x in stage_ms.mean(axis=0)])),
         "compress": {"ms_per_worker": compress_ms, "elements_per_s": total / (compress_ms * 1e-3),
                      "algorithmic_gbs": compress_bytes / (compress_ms * 1e-3) / 1e9,
-                     "frac_of_peak": compress_bytes / (compress_ms * 1e-3) / 1e9 / peak},
+                     "frac_of_peak": compress_bytes / (compress_ms * 1e-3) / 1e9 / peak,
+                     "what": "one dgc_compress alone on one stream (one worker per GPU)"},
         "step": {"algorithmic_bytes": step_bytes, "algorithmic_gbs": step_gbs,
                  "frac_of_peak": step_gbs / peak},
-        "timeline": timeline,
-        "receive": receive, "wire_format": wire, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "cpu_baseline": cpu,
+        "timeline": timeline, "receive": receive, "wire_format": wire, "e2e": e2e,
+        "gpu_launches": int(launches), "clocks": clocks,
     }
+    del pool, out_i, out_v, dense, weights, ws, states
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_1712_01887_b200 import build
+    build.build()
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.cuda.current_device()
+    wl = I.workload(args.workload) if args.workload != "sweep" else I.workload("sweep", n=args.n)
+    if args.clip is not None:
+        wl.clip_threshold = args.clip
+    if args.sparsity is not None:
+        wl.sparsity = args.sparsity
+    head = measure(args, wl, rank, world, dev, headline=True)
+    # the second target workload: the LSTM-shaped set (4 workers, clipping on), same step,
+    # same clocks sampler, device timings only; part of the default run
+    second = None
+    plain = (args.workload == "resnet50" and args.clip is None and args.sparsity is None
+             and args.workers is None)
+    if plain and not args.no_second:
+        w2 = I.workload("lstm")
+        r2 = measure(args, w2, rank, world, dev, headline=False)
+        second = {k: r2[k] for k in ("value", "ms_per_step", "repeats", "config", "roofline",
+                                     "stages_ms", "compress", "step", "receive", "gpu_launches",
+                                     "clocks")}
+        second["unit"] = UNIT
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    cpu = None if args.no_cpu_baseline else cpu_baseline(wl, budget_s=args.cpu_seconds)
+    line = {
+        "metric": METRIC, "value": head["value"], "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": head["ms_per_step"],
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+    }
+    for k in ("config", "repeats", "roofline", "stages_ms", "compress", "step", "timeline",
+              "receive", "wire_format", "e2e", "gpu_launches", "clocks"):
+        line[k] = head[k]
+    line["cpu_baseline"] = cpu
+    if second is not None:
+        line["lstm"] = second
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -457,7 +552,7 @@ def run_ours(args):
 
 # ----------------------------------------------------------------------------- CPU oracle legs
 
-def _oracle_step_factory(wl, n_workers, pool=POOL):
+def _oracle_step_factory(wl, n_workers, pool=E2E_POOL):
     """The same step on the CPU oracle, for `n_workers` simulated workers."""
     from oracle import dgc_oracle as O
     off, L = _layout(wl)
@@ -501,9 +596,10 @@ def cpu_baseline(wl, budget_s=20.0):
 
 
 def run_schedule(args):
-    """The warm-up schedule of Sec. 4.1 on one workload (BASELINE config 4: 5 stages of
-    `--stage-iters` iterations at 75 %, 93.75 %, 98.4375 %, 99.6 %, 99.9 % sparsity): the same
-    step as the headline benchmark, timed per stage, dgc_set_sparsity between stages."""
+    """The warm-up schedule of Sec. 4.1 on one workload (meant for the DeepSpeech-shaped set: 5
+    stages of `--stage-iters` iterations at 75 %, 93.75 %, 98.4375 %, 99.6 %, 99.9 % sparsity):
+    the same step as the headline benchmark, timed per stage, dgc_set_sparsity between stages."""
+    POOL = E2E_POOL
     import torch
     from paper_1712_01887_b200 import build
     build.build()
@@ -579,6 +675,7 @@ def run_schedule(args):
 def run_literal(args):
     """Compress-only timing of the paper-literal sampled selection (select_mode = 1, Sec. 5 as
     stated: variable number of entries, so the fixed-size step of the headline does not apply)."""
+    POOL = E2E_POOL
     import torch
     from paper_1712_01887_b200 import build
     build.build()
@@ -650,7 +747,10 @@ def run_reference(args):
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "tensors": len(wl.shapes), "elements": wl.total,
                    "simulated_workers": nw, "sparsity": wl.sparsity, "momentum": wl.momentum,
-                   "clip_threshold": wl.clip_threshold},
+                   "clip_threshold": wl.clip_threshold,
+                   "sample": f"{nw} of the workload's {wl.num_workers} simulated workers per "
+                             "step (a bounded sample: the metric is per element, the decode "
+                             f"sums {nw} lists instead of {wl.num_workers})"},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
                          "sample": sample, "host_cpus": os.cpu_count()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -687,6 +787,11 @@ def main():
                          "their replays")
     ap.add_argument("--separate-receive", action="store_true",
                     help="decode and SGD as two calls instead of the one-pass entry point")
+    ap.add_argument("--repeats", type=int, default=3,
+                    help="times the timed region of exactly --steps steps is run; the median "
+                         "is reported, all of them listed")
+    ap.add_argument("--no-second", action="store_true",
+                    help="skip the second target workload (LSTM-shaped set) of the default run")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -13,14 +13,12 @@ from oracle import dgc_oracle as O
 from paper_1712_01887_b200 import binding as B
 
 NORM_RTOL = 1e-6          # clipping norm: relative tolerance (fp64 sums in different orders)
-NEAR_THR_RTOL = 1e-6      # |v| this close to the threshold may differ if the clip coefficient did
 
 
 @dataclass
 class ParityReport:
     worker_iterations: int = 0
     coef_overrides: int = 0          # oracle re-run with the GPU's clip coefficient
-    near_threshold_ties: int = 0     # selected-set differences inside NEAR_THR_RTOL of the threshold
     full_select: int = 0             # tensors that took the full-selection path on the GPU
     max_norm_rel_err: float = 0.0
     notes: List[str] = field(default_factory=list)
@@ -87,18 +85,10 @@ class Pair:
         rep.worker_iterations += 1
         rep.full_select += int(st.full_select_last)
         if gi.tobytes() != r.idx.tobytes():
-            # tolerated only for entries within NEAR_THR_RTOL of the threshold (and counted)
+            # With equal clip coefficients (ensured above) the selected set is unique: any
+            # difference is an error, however close the entries are to the threshold.
             diff = np.setxor1d(gi, r.idx)
-            kth, _ = self.gpu.thresholds()
-            v_pre = np.zeros(self.gpu.arena_len, np.float32)
-            v_pre[r.idx] = r.val
-            v_pre[gi] = gv
-            for i in diff:
-                j = int(np.searchsorted(self.gpu.arena_offset, i, side="right") - 1)
-                thr = np.array([kth[j]], np.uint32).view(np.float32)[0]
-                assert abs(abs(v_pre[i]) - thr) <= NEAR_THR_RTOL * thr, (i, v_pre[i], thr)
-            rep.near_threshold_ties += diff.size
-            raise AssertionError(f"selected sets differ at {diff.size} near-threshold entries")
+            raise AssertionError(f"selected sets differ at {diff.size} entries, first {diff[:8]}")
         _assert_bits(gv, r.val, "sent values")
         if check_state:
             u, v = self.gpu.read()

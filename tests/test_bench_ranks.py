@@ -67,6 +67,23 @@ def test_reference_arm_prints_contract_line_and_other_ranks_stay_silent():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["value"] == line["value"]
     assert line["config"]["workload"] == "lstm_small"
+    assert line["config"]["sample"].startswith("2 of the workload's 4 simulated workers")
+
+
+def test_traffic_table_and_gradient_pool_size():
+    """roofline.traffic comes from the committed table of ncu captures (keyed by workload and
+    kernel, None where nothing was captured); the gradient pool has the workload's iteration
+    count."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_1712_01887_b200 import inputs as I
+    t = bench._ncu_traffic("resnet50", "k_update_emit")
+    assert t is not None and 0.5 < t / (20.0 * 25557032) < 1.5
+    assert bench._ncu_traffic("resnet50", "no_such_kernel") is None
+    assert bench._ncu_traffic("cfg1", "k_update_emit") is None
+    assert bench._pool_size(I.workload("resnet50")) == 10
+    assert bench._pool_size(I.workload("lstm")) == 10
+    assert bench._pool_size(I.workload("cfg1")) == 5
 
 
 @pytest.mark.gpu

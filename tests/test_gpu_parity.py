@@ -45,7 +45,6 @@ def _run_workload(P, wl, iterations, workers=None, seed=0, receive=True, schedul
             _, w_host = P.receive_side(lists_i, lists_v, L, w_host, lr=0.1)
     for p in pairs:
         p.close()
-    assert rep.near_threshold_ties == 0
     return rep
 
 
@@ -91,20 +90,28 @@ def test_nesterov_variant_resnet50_no_clip(P):
     _run_workload(P, wl, 2, workers=1, receive=False, nesterov=True)
 
 
-def test_lstm_full_size_one_worker(P):
-    """The 66,034,000-value LSTM-shaped set at full size (15 M-element tensors, 58 parts each):
-    every index, value and state word against the oracle, clipping on."""
+def test_lstm_full_size_all_workers_with_receive_side(P):
+    """The 66,034,000-value LSTM-shaped set at full size (15 M-element tensors, 58 parts each;
+    a row-sparse embedding gradient whose zeros tie in masses): all 4 workers, 3 iterations,
+    clipping on; every index, value and state word against the oracle, then the decoded sum
+    of the 4 lists and the weights after the SGD step."""
     wl = I.workload("lstm")
-    rep = _run_workload(P, wl, 2, workers=1, receive=False)
+    rep = _run_workload(P, wl, 3)
+    assert rep.worker_iterations == 12
     assert rep.full_select == 0
 
 
-def test_deepspeech_full_size_two_warmup_stages(P):
-    """The 122,096,829-value DeepSpeech-shaped set at full size: one iteration at 75 % and
-    one at 99.9 % sparsity (k = 30.5 M and 122 K entries)."""
+def test_deepspeech_full_size_every_warmup_stage(P):
+    """The 122,096,829-value DeepSpeech-shaped set at full size through the whole warm-up
+    schedule of Sec. 4.1 (75 %, 93.75 %, 98.4375 %, 99.6 %, 99.9 %: 30.5 M down to 122 K
+    entries sent), dgc_set_sparsity between the stages; two iterations at 75 % so that the
+    deferred masking of the emission-from-v' path is applied by a following call of the same
+    stage, one in each later stage; receive side included."""
     wl = I.workload("deepspeech")
-    stages = [0.75, 0.999]
-    _run_workload(P, wl, 2, workers=1, receive=False, schedule=lambda t: stages[t])
+    stages = [0.75, 0.75, 0.9375, 0.984375, 0.996, 0.999]
+    rep = _run_workload(P, wl, len(stages), workers=1, schedule=lambda t: stages[t])
+    assert rep.worker_iterations == 6
+    assert rep.full_select == 0
 
 
 @pytest.mark.parametrize("n", [1 << 16, 1 << 18, 1 << 20, 1 << 22, 1 << 24])
@@ -115,10 +122,14 @@ def test_sweep_single_tensor(P, n, sparsity):
     assert rep.full_select == 0
 
 
-@pytest.mark.parametrize("n,sparsity", [(1 << 26, 0.999), (1 << 28, 0.999), (1 << 28, 0.99)])
+@pytest.mark.parametrize("n", [1 << 26, 1 << 28])
+@pytest.mark.parametrize("sparsity", [0.99, 0.999, 0.9999])
 def test_sweep_largest_tensors(P, n, sparsity):
+    """The two largest sizes of the single-tensor sweep at all three sparsities (2 iterations
+    at 2^26, 1 at 2^28 where one oracle iteration takes several seconds)."""
     wl = I.workload("sweep", n=n, sparsity=sparsity)
-    _run_workload(P, wl, 1 if n == 1 << 28 else 2, workers=1, receive=False)
+    rep = _run_workload(P, wl, 1 if n == 1 << 28 else 2, workers=1, receive=False)
+    assert rep.full_select == 0
 
 
 @pytest.mark.parametrize("sparsity", [0.999, 0.99, 0.75, 0.0])
@@ -680,14 +691,16 @@ def test_sparsity_lowered_after_creation_reallocates_scratch(P):
     pair.close()
 
 
-def test_compress_batch_matches_oracle_per_worker(P):
+@pytest.mark.parametrize("clip,T", [(1.0, 3), (0.0, 10)])
+def test_compress_batch_matches_oracle_per_worker(P, clip, T):
     """dgc_compress_batch (what bench.py times): all 8 workers of the ResNet-50-shaped set in
-    one call, with clipping on so that the norm kernels run ahead too; every worker bit for bit
-    against its oracle, then the one-pass receive side."""
+    one call; every worker bit for bit against its oracle, then the one-pass receive side.
+    Once with clipping on (so that the norm kernels run ahead too), and once in the
+    benchmark's own configuration (clipping off) for the 10 iterations the workload states."""
     from oracle import dgc_oracle as O
     from paper_1712_01887_b200 import binding as B
     wl = I.workload("resnet50")
-    NW, T, clip = 8, 3, 1.0
+    NW = 8
     states = [B.State(wl.numel, NW, wl.momentum, clip, wl.sparsity, seed=I.BASE_SEED + w)
               for w in range(NW)]
     L, off = states[0].arena_len, states[0].arena_offset
@@ -716,7 +729,8 @@ def test_compress_batch_matches_oracle_per_worker(P):
             st = states[w].status()
             snap = (oracles[w].u.copy(), oracles[w].v.copy())
             r = oracles[w].compress(hosts[w])
-            assert abs(st.grad_norm - r.norm) <= 1e-6 * r.norm and r.coef < 1.0
+            if clip > 0:
+                assert abs(st.grad_norm - r.norm) <= 1e-6 * r.norm and r.coef < 1.0
             if np.float32(st.clip_coef).tobytes() != np.float32(r.coef).tobytes():
                 oracles[w].u[:], oracles[w].v[:] = snap
                 r = oracles[w].compress(hosts[w], coef_override=st.clip_coef)
@@ -782,7 +796,8 @@ def test_cuda_graph_replay_matches_oracle(P):
             assert st.iterations == t + 1
             snap = (oracles[w].u.copy(), oracles[w].v.copy())
             r = oracles[w].compress(hosts[w])
-            assert abs(st.grad_norm - r.norm) <= 1e-6 * r.norm and r.coef < 1.0
+            if clip > 0:
+                assert abs(st.grad_norm - r.norm) <= 1e-6 * r.norm and r.coef < 1.0
             if np.float32(st.clip_coef).tobytes() != np.float32(r.coef).tobytes():
                 oracles[w].u[:], oracles[w].v[:] = snap
                 r = oracles[w].compress(hosts[w], coef_override=st.clip_coef)
