@@ -46,9 +46,12 @@ LR = 0.01
 TRAFFIC_JSON = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
 
 
-def _pool_size(wl) -> int:
+def _pool_size(wl, override=None) -> int:
     """Distinct pre-generated gradients per worker: the workload's stated iteration count (10
-    for the ResNet-50- and LSTM-shaped sets), so that consecutive steps see fresh gradients."""
+    for the ResNet-50- and LSTM-shaped sets), so that consecutive steps see fresh gradients;
+    --pool overrides it (small profiler captures)."""
+    if override:
+        return max(1, int(override))
     return max(2, min(int(wl.iterations), 10))
 
 
@@ -185,7 +188,7 @@ def measure(args, wl, rank, world, dev, headline):
     from paper_1712_01887_b200 import binding as B
 
     NW = args.workers or wl.num_workers
-    POOL = _pool_size(wl)
+    POOL = _pool_size(wl, args.pool)
     off, L, grads = _host_gradients(wl, NW, rank, POOL)
     total = wl.total
     states = [B.State(wl.numel, wl.num_workers, wl.momentum, wl.clip_threshold, wl.sparsity,
@@ -790,6 +793,9 @@ def main():
     ap.add_argument("--repeats", type=int, default=3,
                     help="times the timed region of exactly --steps steps is run; the median "
                          "is reported, all of them listed")
+    ap.add_argument("--pool", type=int, default=None,
+                    help="distinct gradients per worker (default: the workload's iteration "
+                         "count, at most 10)")
     ap.add_argument("--no-second", action="store_true",
                     help="skip the second target workload (LSTM-shaped set) of the default run")
     ap.add_argument("--e2e-steps", type=int, default=5)

@@ -31,6 +31,7 @@
 // k_sgd (Alg. 4 update line).
 #pragma once
 
+#include <cooperative_groups.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -52,6 +53,9 @@ constexpr int kSelectThreads = 1024;
 constexpr int kSelectBatchThreads = 512;   // k_select in a batch of several workers
 constexpr int kSelectMaxSmemKeys = 51200;
 constexpr int kSelectMaxParts = 256;   // parts of one tensor whose tables fit in shared memory
+constexpr int kClusterSize = 8;        // k_select_cluster: blocks (SMs) that share one tensor
+constexpr int kClusterThreads = 512;
+constexpr int kClusterMinParts = 8;    // tensors of at least this many parts use the whole cluster
 constexpr int kEmitThreads = kPartSegs;   // one thread per segment of the part
 constexpr int kEmitRegs = 8;              // candidates per thread kept in registers
 constexpr int kMaskStride = 17;           // words per segment in the winner bitmaps (16 + 1 pad)
@@ -250,8 +254,35 @@ __device__ __forceinline__ void block_excl_scan2(int a, int b, int* sh, int& ea,
 // of warps, so that the integer atomics of different warps do not collide;
 // they are folded into one of two alternating 256-bin histograms, in which
 // warp 0 finds the digit.  hist: kHistWords(blockDim.x) words of shared
-// memory, sh: 3 words.  blockDim.x is a multiple of 256, at least 512.
+// memory, sh: 3 words.  blockDim.x is a multiple of 256.
 // Returns the key; n_gt = number of keys strictly greater.
+// One warp: in a 256-bin histogram h of digit counts, the digit (from the largest) at which the
+// cumulative count reaches `remaining` -> sh[0]; keys in larger digits -> sh[1]; keys in that
+// digit -> sh[2].
+__device__ __forceinline__ void warp_find_digit(const uint32_t* h, int remaining, int* sh) {
+  const int lane = threadIdx.x & 31;
+  const int hi = 255 - 8 * lane;          // this lane covers bins hi, hi-1, .., hi-7
+  uint32_t loc[8];
+  uint32_t s = 0;
+#pragma unroll
+  for (int q = 0; q < 8; ++q) { loc[q] = h[hi - q]; s += loc[q]; }
+  const uint32_t incl = (uint32_t)warp_incl_scan((int)s);
+  const uint32_t excl = incl - s;
+  if (excl < (uint32_t)remaining && (uint32_t)remaining <= incl) {
+    uint32_t c = excl;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (c + loc[q] >= (uint32_t)remaining) {
+        sh[0] = hi - q;
+        sh[1] = (int)c;
+        sh[2] = (int)loc[q];     // after the last pass: keys equal to the result
+        break;
+      }
+      c += loc[q];
+    }
+  }
+}
+
 __host__ __device__ constexpr int kHistCopies(int threads) { return threads / 32 < 16 ? threads / 32 : 16; }
 __host__ __device__ constexpr int kHistWords(int threads) { return kHistCopies(threads) * 257 + 512; }
 
@@ -299,29 +330,10 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
       __syncthreads();
     }
     if (tid < 32) {
-      const uint32_t* h = folded + cur * 256;
-      const int hi = 255 - 8 * lane;          // this lane covers bins hi, hi-1, .., hi-7
-      uint32_t loc[8];
-      uint32_t s = 0;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) { loc[q] = h[hi - q]; s += loc[q]; }
-      const uint32_t incl = (uint32_t)warp_incl_scan((int)s);
-      const uint32_t excl = incl - s;
-      if (excl < (uint32_t)remaining && (uint32_t)remaining <= incl) {
-        uint32_t c = excl;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          if (c + loc[q] >= (uint32_t)remaining) {
-            sh[0] = hi - q;
-            sh[1] = (int)c;
-            sh[2] = (int)loc[q];     // after the last pass: keys equal to the result
-            break;
-          }
-          c += loc[q];
-        }
-      }
-    } else if (tid < 288) {
-      folded[(cur ^ 1) * 256 + tid - 32] = 0;   // clear the other histogram for the next pass
+      warp_find_digit(folded + cur * 256, remaining, sh);
+    } else {
+      // the other warps clear the other histogram for the next pass
+      for (int i = tid - 32; i < 256; i += nt - 32) folded[(cur ^ 1) * 256 + i] = 0;
     }
     __syncthreads();
     prefix |= (uint32_t)sh[0] << shift;
@@ -422,6 +434,8 @@ k_sumsq(Plan p, const float* __restrict__ g, double thr_local, int clip_on) {
 // draws of single elements, draw r of tensor j at floor(h n / 2^64), h = mix64(call seed xor
 // (j << 32) xor r); a thread takes draws 4s .. 4s + 3.  Draws beyond `samples` count as key 0,
 // which cannot move the rank-th largest key (rank <= samples).
+// (Capping the registers at 32 for a fourth block per SM was measured: the spills cost more
+// than the slot gains, 0.776 -> 0.785 ms per batched step.)
 template <bool CLIP, bool NEST, bool LITERAL>
 __global__ void __launch_bounds__(kSampleThreads)
 k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_base) {
@@ -430,7 +444,10 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   // hashed, so that consecutive calls draw unrelated positions
   const uint64_t call_seed = mix64(seed_base + (uint64_t)__ldcg(p.iter));
   __shared__ uint32_t hist[kHistWords(kSampleThreads)];
-  __shared__ uint32_t surv[kSampleSurvivors];
+  // the survivors share the private histogram copies' words: wherever survivors are kept the
+  // selections run without private copies (only the last 512 words of hist are in use)
+  uint32_t* surv = hist;
+  static_assert(kSampleSurvivors <= kHistCopies(kSampleThreads) * 257, "survivors alias the copies");
   __shared__ int sh[3];
   __shared__ int s_cnt;
   __shared__ uint32_t s_max;
@@ -897,30 +914,34 @@ __device__ __forceinline__ bool tie_fill_parts(const Plan& p, int p0, int pn, in
 // THREADS: 1024 for a call that runs alone (shortest chain for the largest tensor), 512 when
 // several workers' selections run together (twice the blocks per SM: the batch's tail is
 // bound by block slots, not by one block's chain).
+// Shared memory of one selection block besides the dynamic [histograms | keys] area.
+struct SelectShared {
+  int sh[66];
+  int flag;
+  uint32_t max;
+  int pbase[kSelectMaxParts + 1];   // first key of each part in the compact order
+  int pcb[kSelectMaxParts];         // start of each part's candidate list
+  int gt[kSelectMaxParts];
+  int eq[kSelectMaxParts];
+};
+
+// The selection of tensor j by one block of THREADS threads (the whole of k_select, and what
+// k_select_cluster does for tensors that one block handles).
 template <int THREADS>
-__global__ void __launch_bounds__(THREADS)
-k_select(Plan p, int smem_keys) {
-  pdl_enter();
-  timeline_mark(p.timeline, 2);
-  const int parity = (int)(__ldcg(p.iter) & 1);
-  extern __shared__ uint32_t dyn_smem[];          // [histograms | keys]
+__device__ __forceinline__ void select_tensor(const Plan& p, int j, const TensorMeta& t,
+                                              int smem_keys, int parity, uint32_t* dyn_smem,
+                                              SelectShared& S) {
   uint32_t* hist = dyn_smem;
   uint32_t* skeys = dyn_smem + kHistWords(THREADS);
-  __shared__ int sh[66];
-  __shared__ int s_flag;
-  __shared__ uint32_t s_max;
-  __shared__ int s_pbase[kSelectMaxParts + 1];   // first key of each part in the compact order
-  __shared__ int s_pcb[kSelectMaxParts];         // start of each part's candidate list
-  __shared__ int s_gt[kSelectMaxParts];
-  __shared__ int s_eq[kSelectMaxParts];
-  const int j = blockIdx.x;
+  int* sh = S.sh;
+  int& s_flag = S.flag;
+  uint32_t& s_max = S.max;
+  int* s_pbase = S.pbase;
+  int* s_pcb = S.pcb;
+  int* s_gt = S.gt;
+  int* s_eq = S.eq;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const TensorMeta t = load_record(p.tm + j);
   const int p0 = t.part_first, pn = t.part_num, k = t.k;
-  if (j == 0 && tid < 4) p.diag[(parity ^ 1) * 4 + tid] = 0;   // next call's counters
-  // k_big_* select the big tensors, which include every tensor of more than kSelectMaxParts
-  // parts: the per-part tables below always fit
-  if (t.big || pn > kSelectMaxParts) return;
   if (tid == 0) { s_flag = 0; s_max = 0u; }
   __syncthreads();
   // candidates per part (one load round for all parts), overflow check, compact bases
@@ -1127,6 +1148,220 @@ k_select(Plan p, int smem_keys) {
     p.t_nnz[j] = nnz;
     atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
   }
+}
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
+k_select(Plan p, int smem_keys) {
+  pdl_enter();
+  timeline_mark(p.timeline, 2);
+  const int parity = (int)(__ldcg(p.iter) & 1);
+  extern __shared__ uint32_t dyn_smem[];          // [histograms | keys]
+  __shared__ SelectShared S;
+  const int j = blockIdx.x;
+  const TensorMeta t = load_record(p.tm + j);
+  if (j == 0 && threadIdx.x < 4) p.diag[(parity ^ 1) * 4 + threadIdx.x] = 0;   // next call's counters
+  // k_big_* select the big tensors, which include every tensor of more than kSelectMaxParts
+  // parts: the per-part tables always fit
+  if (t.big || t.part_num > kSelectMaxParts) return;
+  select_tensor<THREADS>(p, j, t, smem_keys, parity, dyn_smem, S);
+}
+
+// The same selection with a thread-block cluster per tensor: kClusterSize blocks on as many SMs
+// share the candidates of one tensor (a contiguous range of its parts each) and exchange their
+// digit histograms through distributed shared memory, so that the longest chain of the tail --
+// the tensor with the most candidates -- is cut several times over: one block spends about
+// 120 instructions per candidate, 41 us for the 30 K candidates of a 15 M-element tensor.
+// Tensors of fewer than kClusterMinParts parts, and every case that needs no key (tie-fill,
+// full selection, paper-literal pass-through), are handled by the cluster's first block alone;
+// the other blocks leave at once.  Every decision that steers the cluster barriers is taken
+// from values all blocks read alike (plan tables, the parts' counts), so that all blocks of a
+// cluster pass the same barriers.
+struct ClusterShared {
+  uint32_t hist[2][256];   // this block's digit counts, current and next pass
+  uint32_t folded[256];    // the cluster's digit counts
+  uint32_t max;
+};
+
+template <int THREADS>
+__global__ void __launch_bounds__(THREADS)
+k_select_cluster(Plan p, int smem_keys) {
+  namespace cg = cooperative_groups;
+  pdl_enter();
+  timeline_mark(p.timeline, 2);
+  cg::cluster_group cluster = cg::this_cluster();
+  const int r = (int)cluster.block_rank();
+  const int parity = (int)(__ldcg(p.iter) & 1);
+  extern __shared__ uint32_t dyn_smem[];          // [histograms | keys]
+  __shared__ SelectShared S;
+  __shared__ ClusterShared X;
+  const int j = blockIdx.x / kClusterSize;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const TensorMeta t = load_record(p.tm + j);
+  const int p0 = t.part_first, pn = t.part_num, k = t.k;
+  if (blockIdx.x == 0 && tid < 4) p.diag[(parity ^ 1) * 4 + tid] = 0;   // next call's counters
+  if (t.big || pn > kSelectMaxParts) return;                 // (same for the whole cluster)
+  if (pn < kClusterMinParts) {
+    if (r == 0) select_tensor<THREADS>(p, j, t, smem_keys, parity, dyn_smem, S);
+    return;
+  }
+  static_assert(kSelectMaxParts <= THREADS, "one thread per part");
+  // every block for itself: candidates per part, overflow, compact bases of all parts
+  if (tid == 0) { S.flag = 0; X.max = 0u; }
+  __syncthreads();
+  {
+    int c = 0;
+    if (tid < pn) {
+      const PartMeta pm = load_record(p.pm + p0 + tid);
+      c = __ldcg(p.p_count + p0 + tid);
+      if (c > pm.cap) S.flag = 1;
+      S.pcb[tid] = pm.cbase;
+    }
+    int ex, e2, tot, t2;
+    block_excl_scan2(c, 0, S.sh, ex, e2, tot, t2);
+    if (tid < pn) S.pbase[tid] = ex;
+    if (tid == 0) S.pbase[pn] = tot;
+  }
+  __syncthreads();
+  const int total = S.pbase[pn];
+  const bool overflow = S.flag != 0;
+  const bool literal = p.literal != 0;
+  if (overflow || (!literal && total < k) || (literal && total <= 2 * k)) {
+    // no exact selection among the candidates: one block does what there is to do
+    __syncthreads();
+    if (r == 0) select_tensor<THREADS>(p, j, t, smem_keys, parity, dyn_smem, S);
+    return;
+  }
+  // ---- the whole cluster: this block takes parts [q0, q1)
+  uint32_t* skeys = dyn_smem;
+  const int q0 = r * pn / kClusterSize, q1 = (r + 1) * pn / kClusterSize;
+  const int m0 = S.pbase[q0], m = S.pbase[q1] - m0;
+  const bool in_smem = m <= smem_keys;
+  const int myparts = q1 - q0;
+  const int slices = myparts > 0 ? max(1, (THREADS / 32) / myparts) : 1;
+  if (in_smem) {
+    uint32_t tmax = 0;
+    for (int unit = warp; unit < myparts * slices; unit += THREADS / 32) {
+      const int q = q0 + unit / slices, sl = unit % slices;
+      const int b0 = S.pbase[q] - m0, c = S.pbase[q + 1] - S.pbase[q];
+      const float* src = p.cand_val + S.pcb[q];
+#pragma unroll 4
+      for (int i = sl * 32 + lane; i < c; i += slices * 32) {
+        const uint32_t key = mag_key(__ldcg(src + i));
+        skeys[b0 + i] = key;
+        tmax = max(tmax, key);
+      }
+    }
+    const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
+    if (lane == 0 && wmax) atomicMax(&X.max, wmax);
+  } else if (tid == 0) {
+    X.max = 0x7FFFFFFFu;                           // (keys stay in global memory: no maximum)
+  }
+  for (int i = tid; i < 512; i += THREADS) (&X.hist[0][0])[i] = 0u;
+  __syncthreads();
+  cluster.sync();
+  uint32_t kmax = 0u;
+#pragma unroll
+  for (int rr = 0; rr < kClusterSize; ++rr) kmax = max(kmax, *cluster.map_shared_rank(&X.max, rr));
+  const uint32_t kbase = __ldcg(p.p_thr + p0);     // every candidate reached the proposal
+  // my keys, from shared or (a share that does not fit) from global memory
+  auto each = [&](auto f) {
+    if (in_smem) {
+      for (int i = tid; i < m; i += THREADS) f(skeys[i]);
+    } else {
+      for (int q = q0; q < q1; ++q) {
+        const int c = S.pbase[q + 1] - S.pbase[q];
+        const float* src = p.cand_val + S.pcb[q];
+        for (int i = tid; i < c; i += THREADS) f(mag_key(__ldcg(src + i)));
+      }
+    }
+  };
+  // radix select over the bits in which kmax - kbase can differ, 8 per pass: local counts,
+  // cluster barrier, every block folds the eight histograms and finds the same digit
+  const uint32_t span = kmax - kbase;
+  const int passes = span == 0 ? 0 : (32 - __clz(span) + 7) / 8;
+  uint32_t prefix = 0, mask = 0;
+  int remaining = k;
+  int cur = 0;
+  for (int shift = 8 * (passes - 1); shift >= 0; shift -= 8, cur ^= 1) {
+    each([&](uint32_t key) {
+      key -= kbase;
+      if ((key & mask) == prefix) atomicAdd(&X.hist[cur][(key >> shift) & 255u], 1u);
+    });
+    __syncthreads();
+    cluster.sync();
+    if (tid < 256) {
+      uint32_t sum = 0;
+#pragma unroll
+      for (int rr = 0; rr < kClusterSize; ++rr) sum += *cluster.map_shared_rank(&X.hist[cur][tid], rr);
+      X.folded[tid] = sum;
+    } else if (tid < 512) {
+      // next pass's counts start from zero (the others read this buffer a pass ago and have
+      // passed the barrier above since)
+      X.hist[cur ^ 1][tid - 256] = 0u;
+    }
+    __syncthreads();
+    if (tid < 32) warp_find_digit(X.folded, remaining, S.sh);
+    __syncthreads();
+    prefix |= (uint32_t)S.sh[0] << shift;
+    mask |= 255u << shift;
+    remaining -= S.sh[1];
+    __syncthreads();
+  }
+  static_assert(THREADS >= 512, "threads 256..511 clear the next pass's histogram");
+  const uint32_t kth = kbase + prefix;
+  const int n_gt = k - remaining;
+  // per part of mine: candidates above and tied with the k-th key
+  for (int q = q0 + tid; q < q1; q += THREADS) { S.gt[q] = 0; S.eq[q] = 0; }
+  __syncthreads();
+  for (int unit = warp; unit < myparts * slices; unit += THREADS / 32) {
+    const int q = q0 + unit / slices, sl = unit % slices;
+    const int b0 = S.pbase[q] - m0, c = S.pbase[q + 1] - S.pbase[q];
+    const float* src = p.cand_val + S.pcb[q];
+    int gt = 0, eq = 0;
+    for (int i = sl * 32 + lane; i < c; i += slices * 32) {
+      const uint32_t key = in_smem ? skeys[b0 + i] : mag_key(__ldcg(src + i));
+      gt += key > kth;
+      eq += key == kth;
+    }
+    gt = __reduce_add_sync(0xFFFFFFFFu, gt);
+    eq = __reduce_add_sync(0xFFFFFFFFu, eq);
+    if (lane == 0) {
+      if (gt) atomicAdd(&S.gt[q], gt);
+      if (eq) atomicAdd(&S.eq[q], eq);
+    }
+  }
+  __syncthreads();
+  cluster.sync();
+  if (r == 0) {
+    // the first block collects every part's counts from its owner and places the parts
+    const int quota = k - n_gt;                    // ties with kth to send, lowest indices first
+    const int out_off = literal ? 0 : t.out_off;   // paper-literal: k_emit_mask adds the tensor's base
+    int gt = 0, eq = 0;
+    if (tid < pn) {
+      int owner = 0;
+      while ((owner + 1) * pn / kClusterSize <= tid) ++owner;
+      gt = *cluster.map_shared_rank(&S.gt[tid], owner);
+      eq = *cluster.map_shared_rank(&S.eq[tid], owner);
+    }
+    int bg, be, tg, te;
+    block_excl_scan2(gt, eq, S.sh, bg, be, tg, te);
+    if (tid < pn) {
+      PartSel ps;
+      ps.kth = kth;
+      ps.quota = max(0, min(quota - be, eq));
+      ps.out_base = out_off + bg + min(be, quota);
+      ps.dense = 0;
+      p.psel[p0 + tid] = ps;
+    }
+    if (tid == 0) {
+      p.t_kth[j] = kth;
+      p.t_cand[j] = total;
+      p.t_nnz[j] = k;
+      atomicAdd((unsigned long long*)&p.diag[parity * 4 + 2], (unsigned long long)total);
+    }
+  }
+  cluster.sync();      // the others' shared memory stays until the first block has read it
 }
 
 // ------------------------------------------------------------------ K4b: multi-block exact k-th key
