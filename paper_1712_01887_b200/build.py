@@ -20,7 +20,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
             and all(os.path.getmtime(LIB) >= os.path.getmtime(d) for d in deps)):
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
+    extra = os.environ.get("NVCC_EXTRA_FLAGS", "").split()      # e.g. -D switches of variants
+    cmd = [nvcc] + NVCC_FLAGS + extra + (["-Xptxas", "-v"] if verbose else []) + \
           ["-I", INCLUDE, "-o", LIB, SRC]
     subprocess.run(cmd, check=True)
     return LIB

@@ -269,6 +269,12 @@ void build_host_plan(dgc_state* st, double sparsity) {
     if (!big) st->max_inblock_parts = std::max<int>(st->max_inblock_parts, (int)nparts);
     pos += nseg * kSeg;
   }
+  // sampling blocks of the tensors with the most blocks first: their last block, which selects
+  // among all of them, ends the kernel (a tensor's blocks stay together and in chunk order)
+  std::stable_sort(st->sample_blocks.begin(), st->sample_blocks.end(),
+                   [&](const SampleBlock& a, const SampleBlock& b) {
+                     return st->tm[a.tensor].chunks > st->tm[b.tensor].chunks;
+                   });
   st->arena_len = pos;
   st->max_nnz = out;
   st->cand_total = cbase;

