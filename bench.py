@@ -390,8 +390,11 @@ def measure(args, wl, rank, world, dev, headline):
         KE = max(1, min(K, args.e2e_steps))
 
         def e2e_step(t):
-            for w in range(NW):
-                states[w].compress_host(hosts[w][t % E2E_POOL], hi[w], hv[w])
+            if args.no_batch:
+                for w in range(NW):
+                    states[w].compress_host(hosts[w][t % E2E_POOL], hi[w], hv[w])
+            else:
+                B.compress_host_batch(states, [hosts[w][t % E2E_POOL] for w in range(NW)], hi, hv)
             # the lists a receiver would get are on the host now; the receive side runs on the
             # device copies the call also left in the state's output staging
             for w in range(NW):

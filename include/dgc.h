@@ -179,6 +179,19 @@ int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
 int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_idx_host,
                           float* out_val_host, int64_t capacity, void* stream);
 
+/* dgc_compress_host for several workers of one GPU (the same iteration of Algorithm 4 for each,
+ * Sec. 3.2, Eq. 5, Sec. 3.3, Sec. 5): every worker's gradient is copied from host memory, its
+ * call runs, and its dgc_max_nnz pairs are copied back, each worker on its own internal stream,
+ * so that one worker's kernels run while the next worker's gradient is still crossing the bus.
+ * Same results as dgc_compress_host per state.  Host arrays [num_states] of host pointers
+ * (pinned memory makes the copies asynchronous); capacity[w] >= dgc_max_nnz(states[w]).
+ * Synchronises `stream` before returning: the lists are valid on return.  Not for stream
+ * capture (it allocates staging on first use and synchronises). */
+int32_t dgc_compress_host_batch(int32_t num_states, dgc_state* const* states,
+                                const float* const* grads_host, int32_t* const* out_idx_host,
+                                float* const* out_val_host, const int64_t* capacity,
+                                void* stream);
+
 /* Algorithm 4, line "G_t <- sum_k encode(G~_t^k)", for N workers' lists that
  * already sit in this GPU's memory: dense_out[i] = (((+0 + val_0) + val_1) ...)
  * over the workers that list index i, in worker order, fp32; +0 elsewhere.

@@ -60,6 +60,9 @@ _sigs = {
                                             ctypes.POINTER(_vp), ctypes.POINTER(_vp),
                                             ctypes.POINTER(_vp), _i64p, _vp]),
     "dgc_compress_host": (ctypes.c_int32, [_vp, _vp, _vp, _vp, ctypes.c_int64, _vp]),
+    "dgc_compress_host_batch": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
+                                                 ctypes.POINTER(_vp), ctypes.POINTER(_vp),
+                                                 ctypes.POINTER(_vp), _i64p, _vp]),
     "dgc_decode_accumulate": (ctypes.c_int32, [ctypes.c_int32, ctypes.POINTER(_vp),
                                                ctypes.POINTER(_vp), _i64p, _vp, ctypes.c_int64,
                                                _vp, ctypes.c_int64, _vp]),
@@ -279,6 +282,27 @@ def compress_batch(states: Sequence["State"], grads: Sequence[torch.Tensor],
         if g.numel() != st.arena_len:
             raise ValueError("gradient arena has the wrong length")
     _check(_lib.dgc_compress_batch(n, sp, gp, ip, vp, cap, _stream(stream)), "dgc_compress_batch")
+
+
+def compress_host_batch(states: Sequence["State"], grads: Sequence[torch.Tensor],
+                        out_idx: Sequence[torch.Tensor], out_val: Sequence[torch.Tensor],
+                        stream=None) -> None:
+    """dgc_compress_host for several workers on one GPU: host gradients in, host lists out,
+    the workers' copies and kernels overlapped; the lists are valid on return."""
+    n = len(states)
+    for st, g, a, b in zip(states, grads, out_idx, out_val):
+        for t, dt in ((g, torch.float32), (a, torch.int32), (b, torch.float32)):
+            if t.is_cuda or t.dtype != dt or not t.is_contiguous():
+                raise ValueError("expected contiguous host tensors")
+        if g.numel() != st.arena_len:
+            raise ValueError("gradient arena has the wrong length")
+    sp = (_vp * n)(*[st._h for st in states])
+    gp = (_vp * n)(*[g.data_ptr() for g in grads])
+    ip = (_vp * n)(*[t.data_ptr() for t in out_idx])
+    vp = (_vp * n)(*[t.data_ptr() for t in out_val])
+    cap = (ctypes.c_int64 * n)(*[min(a.numel(), b.numel()) for a, b in zip(out_idx, out_val)])
+    _check(_lib.dgc_compress_host_batch(n, sp, gp, ip, vp, cap, _stream(stream)),
+           "dgc_compress_host_batch")
 
 
 def decode_workspace_bytes(num_workers: int, dense_len: int) -> int:

@@ -710,20 +710,13 @@ BatchResources g_batch[64];
 std::mutex g_batch_mutex;
 }  // namespace
 
-int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
-                           const float* const* grad_arenas, int32_t* const* out_idx,
-                           float* const* out_val, const int64_t* capacity, void* stream) {
-  if (num_states < 1 || !states || !grad_arenas || !out_idx || !out_val || !capacity)
-    return DGC_EINVAL;
-  for (int w = 0; w < num_states; ++w) {
-    dgc_state* st = states[w];
-    if (!st || !st->alive || st->broken) return DGC_ESTATE;
-    if (st->device != states[0]->device) return DGC_EINVAL;
-    if (!grad_arenas[w] || !out_idx[w] || !out_val[w]) return DGC_EINVAL;
-    if ((reinterpret_cast<uintptr_t>(grad_arenas[w]) & 15u) != 0) return DGC_EINVAL;
-    if (capacity[w] < st->max_nnz) return DGC_ECAPACITY;
-    for (int x = 0; x < w; ++x) if (states[x] == st) return DGC_EINVAL;
-  }
+// Shared by dgc_compress_batch (device buffers) and dgc_compress_host_batch (host buffers:
+// `host` = true, every worker's gradient is copied into its state's staging first and its lists
+// are copied out afterwards, on the worker's side stream, so that one worker's kernels run under
+// the next worker's copy).
+static int32_t batch_enqueue(int32_t num_states, dgc_state* const* states,
+                             const float* const* grads, int32_t* const* out_idx,
+                             float* const* out_val, cudaStream_t s, bool host) {
   const int dev = states[0]->device;
   if (dev < 0 || dev >= 64) return DGC_EINVAL;
   std::lock_guard<std::mutex> lock(g_batch_mutex);
@@ -736,7 +729,6 @@ int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
     DGC_CUDA(cudaEventCreateWithFlags(&r.fork, cudaEventDisableTiming));
     r.ready = true;
   }
-  cudaStream_t s = as_stream(stream);
   const int used = std::min<int>(num_states, kBatchStreams);
   int32_t rc;
   // Fork: the workers' calls go round robin over the side streams.  Measured on the
@@ -749,10 +741,26 @@ int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
   for (int w = 0; w < num_states && rc == DGC_OK; ++w) {
     cudaStream_t q = r.side[w % kBatchStreams];
     dgc_state* st = states[w];
-    if ((rc = enqueue_head(st, grad_arenas[w], q, nullptr)) != DGC_OK) break;
-    if ((rc = enqueue_stream_pass(st, grad_arenas[w], q)) != DGC_OK) break;
-    if ((rc = enqueue_tail(st, out_idx[w], out_val[w], q, nullptr, num_states >= 4)) != DGC_OK) break;
+    const float* g = grads[w];
+    int32_t* oi = out_idx[w];
+    float* ov = out_val[w];
+    if (host) {
+      if (cudaMemcpyAsync(st->d_stage_g, grads[w], (size_t)st->arena_len * 4,
+                          cudaMemcpyHostToDevice, q) != cudaSuccess) { rc = DGC_ECUDA; break; }
+      g = st->d_stage_g;
+      oi = st->d_stage_idx;
+      ov = st->d_stage_val;
+    }
+    if ((rc = enqueue_head(st, g, q, nullptr)) != DGC_OK) break;
+    if ((rc = enqueue_stream_pass(st, g, q)) != DGC_OK) break;
+    if ((rc = enqueue_tail(st, oi, ov, q, nullptr, num_states >= 4)) != DGC_OK) break;
     st->iterations += 1;
+    if (host) {
+      if (cudaMemcpyAsync(out_idx[w], oi, (size_t)st->max_nnz * 4, cudaMemcpyDeviceToHost, q) !=
+              cudaSuccess ||
+          cudaMemcpyAsync(out_val[w], ov, (size_t)st->max_nnz * 4, cudaMemcpyDeviceToHost, q) !=
+              cudaSuccess) { rc = DGC_ECUDA; break; }
+    }
   }
   // Join, also after an enqueue error: the side streams were forked from the caller's stream
   // (inside a capture they belong to it) and what was enqueued on them must be ordered before
@@ -764,17 +772,38 @@ int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
       if (rc == DGC_OK) rc = DGC_ECUDA;
     }
   }
+  if (rc != DGC_OK) (void)cudaGetLastError();
   return rc;
 }
 
-int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_idx_host,
-                          float* out_val_host, int64_t capacity, void* stream) {
-  if (!st || !st->alive || st->broken) return DGC_ESTATE;
-  if (!grad_host || !out_idx_host || !out_val_host) return DGC_EINVAL;
-  if (capacity < st->max_nnz) return DGC_ECAPACITY;
-  DeviceGuard guard(st->device);
-  if (!guard.ok) return DGC_ECUDA;
-  cudaStream_t s = as_stream(stream);
+static int32_t batch_check(int32_t num_states, dgc_state* const* states, const void* const* a,
+                           const void* const* b, const void* const* c, const int64_t* capacity,
+                           bool aligned16) {
+  if (num_states < 1 || !states || !a || !b || !c || !capacity) return DGC_EINVAL;
+  for (int w = 0; w < num_states; ++w) {
+    dgc_state* st = states[w];
+    if (!st || !st->alive || st->broken) return DGC_ESTATE;
+    if (st->device != states[0]->device) return DGC_EINVAL;
+    if (!a[w] || !b[w] || !c[w]) return DGC_EINVAL;
+    if (aligned16 && (reinterpret_cast<uintptr_t>(a[w]) & 15u) != 0) return DGC_EINVAL;
+    if (capacity[w] < st->max_nnz) return DGC_ECAPACITY;
+    for (int x = 0; x < w; ++x) if (states[x] == st) return DGC_EINVAL;
+  }
+  return DGC_OK;
+}
+
+int32_t dgc_compress_batch(int32_t num_states, dgc_state* const* states,
+                           const float* const* grad_arenas, int32_t* const* out_idx,
+                           float* const* out_val, const int64_t* capacity, void* stream) {
+  const int32_t rc = batch_check(num_states, states, (const void* const*)grad_arenas,
+                                 (const void* const*)out_idx, (const void* const*)out_val,
+                                 capacity, true);
+  if (rc != DGC_OK) return rc;
+  return batch_enqueue(num_states, states, grad_arenas, out_idx, out_val, as_stream(stream), false);
+}
+
+// Device staging of the host-buffer entry points (gradient in, lists out), allocated on first use.
+static int32_t ensure_staging(dgc_state* st) {
   int32_t rc;
   void* ptr = nullptr;
   if (!st->d_stage_g) {
@@ -791,6 +820,19 @@ int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_id
     st->d_stage_val = (float*)ptr;
     st->stage_nnz = st->max_nnz;
   }
+  return DGC_OK;
+}
+
+int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_idx_host,
+                          float* out_val_host, int64_t capacity, void* stream) {
+  if (!st || !st->alive || st->broken) return DGC_ESTATE;
+  if (!grad_host || !out_idx_host || !out_val_host) return DGC_EINVAL;
+  if (capacity < st->max_nnz) return DGC_ECAPACITY;
+  DeviceGuard guard(st->device);
+  if (!guard.ok) return DGC_ECUDA;
+  cudaStream_t s = as_stream(stream);
+  int32_t rc;
+  if ((rc = ensure_staging(st)) != DGC_OK) return rc;
   DGC_CUDA(cudaMemcpyAsync(st->d_stage_g, grad_host, (size_t)st->arena_len * 4,
                            cudaMemcpyHostToDevice, s));
   rc = dgc_compress(st, st->d_stage_g, st->d_stage_idx, st->d_stage_val, st->stage_nnz, stream);
@@ -801,6 +843,25 @@ int32_t dgc_compress_host(dgc_state* st, const float* grad_host, int32_t* out_id
                            cudaMemcpyDeviceToHost, s));
   DGC_CUDA(cudaStreamSynchronize(s));
   return DGC_OK;
+}
+
+int32_t dgc_compress_host_batch(int32_t num_states, dgc_state* const* states,
+                                const float* const* grads_host, int32_t* const* out_idx_host,
+                                float* const* out_val_host, const int64_t* capacity,
+                                void* stream) {
+  int32_t rc = batch_check(num_states, states, (const void* const*)grads_host,
+                           (const void* const*)out_idx_host, (const void* const*)out_val_host,
+                           capacity, false);
+  if (rc != DGC_OK) return rc;
+  DeviceGuard guard(states[0]->device);
+  if (!guard.ok) return DGC_ECUDA;
+  for (int w = 0; w < num_states; ++w)
+    if ((rc = ensure_staging(states[w])) != DGC_OK) return rc;
+  cudaStream_t s = as_stream(stream);
+  rc = batch_enqueue(num_states, states, grads_host, out_idx_host, out_val_host, s, true);
+  const cudaError_t e = cudaStreamSynchronize(s);      // the lists are valid on return
+  if (e != cudaSuccess) { (void)cudaGetLastError(); if (rc == DGC_OK) rc = DGC_ECUDA; }
+  return rc;
 }
 
 }  // extern "C"

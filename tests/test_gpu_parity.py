@@ -367,6 +367,38 @@ def test_compress_host_matches_device_path(P):
     b.close()
 
 
+def test_compress_host_batch_matches_per_worker_calls(P):
+    """dgc_compress_host_batch (what the benchmark's end-to-end leg calls): host gradients of
+    several workers in, host lists out, bit for bit what dgc_compress gives each worker on the
+    device, over three iterations (state carried); more workers than internal streams."""
+    from paper_1712_01887_b200 import binding as B
+    numel = [300000, 70001, 64, 9000]
+    NW = 10
+    rng = np.random.default_rng(16)
+    dev_states = [B.State(numel, NW, 0.9, 1.0, 0.999, seed=w) for w in range(NW)]
+    host_states = [B.State(numel, NW, 0.9, 1.0, 0.999, seed=w) for w in range(NW)]
+    L, nnz = dev_states[0].arena_len, dev_states[0].max_nnz
+    hi = [torch.empty(nnz, dtype=torch.int32).pin_memory() for _ in range(NW)]
+    hv = [torch.empty(nnz, dtype=torch.float32).pin_memory() for _ in range(NW)]
+    for t in range(3):
+        gh = [torch.from_numpy(rng.standard_normal(L).astype(np.float32)).pin_memory()
+              for _ in range(NW)]
+        B.compress_host_batch(host_states, gh, hi, hv)
+        for w in range(NW):
+            oi = torch.empty(nnz, dtype=torch.int32, device="cuda")
+            ov = torch.empty(nnz, dtype=torch.float32, device="cuda")
+            dev_states[w].compress(gh[w].cuda(), oi, ov)
+            assert torch.equal(oi.cpu(), hi[w]), (t, w)
+            assert torch.equal(ov.cpu().view(torch.int32), hv[w].view(torch.int32)), (t, w)
+    ua, va = dev_states[3].read()
+    ub, vb = host_states[3].read()
+    assert ua.tobytes() == ub.tobytes() and va.tobytes() == vb.tobytes()
+    with pytest.raises(B.DgcError):                      # the same state twice
+        B.compress_host_batch([host_states[0], host_states[0]], gh[:2], hi[:2], hv[:2])
+    for st in dev_states + host_states:
+        st.close()
+
+
 def test_abi_errors(P):
     from paper_1712_01887_b200 import binding as B
     with pytest.raises(B.DgcError) as e:
