@@ -204,6 +204,43 @@ void dgc_oracle_compress(int32_t num_tensors, const int64_t* offset, const int64
   }
 }
 
+// The same iteration with clipping per tensor (an option beside the paper's reading, which
+// clips by one norm over the whole set: Sec. 3.2 speaks of "their L2-norms", Appendix C of one
+// ||G^k||_2).  Tensor j is rescaled by coef_j = thr_local / ||g[j]||_2 iff ||g[j]||_2 >
+// thr_local, thr_local = thr_G N^-1/2 as before; everything after the clipping is unchanged.
+//   coef_override : NULL, or one coefficient per tensor that replaces the computed ones
+//   norms_out, coefs_out : per tensor, the computed norm and the coefficient used
+void dgc_oracle_compress_clip_per_tensor(int32_t num_tensors, const int64_t* offset,
+                                         const int64_t* numel, const int64_t* k,
+                                         const int64_t* out_offset, float* u, float* v,
+                                         const float* g, float momentum, double clip_threshold,
+                                         int32_t num_workers, const float* coef_override,
+                                         int32_t brute_force, int32_t nesterov, int32_t* out_idx,
+                                         float* out_val, double* norms_out, float* coefs_out) {
+  std::vector<int64_t> sel;
+  for (int32_t j = 0; j < num_tensors; ++j) {
+    // clip this tensor by its own norm, then Eq. 5 on it
+    double norm = 0.0;
+    float coef = 1.0f;
+    dgc_oracle_clip_coef(1, offset + j, numel + j, g, clip_threshold, num_workers, &norm, &coef);
+    if (coef_override) coef = coef_override[j];
+    norms_out[j] = norm;
+    coefs_out[j] = coef;
+    dgc_oracle_momentum_correction(1, offset + j, numel + j, u, v, g, momentum, coef, nesterov);
+    // select, emit, mask: as in dgc_oracle_compress
+    const int64_t o = offset[j];
+    sel.assign(static_cast<size_t>(k[j]), 0);
+    dgc_oracle_select_topk(numel[j], v + o, k[j], sel.data(), brute_force);
+    for (int64_t r = 0; r < k[j]; ++r) {
+      const int64_t i = o + sel[static_cast<size_t>(r)];
+      out_idx[out_offset[j] + r] = static_cast<int32_t>(i);
+      out_val[out_offset[j] + r] = v[i];
+      v[i] = 0.0f;
+      u[i] = 0.0f;
+    }
+  }
+}
+
 // Algorithm 4, aggregation line: G = sum over workers of their sparse
 // gradients, added in worker order starting from +0.0f.
 void dgc_oracle_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lists,

@@ -59,6 +59,11 @@ def lib() -> ctypes.CDLL:
                                           _f32p, ctypes.c_float, ctypes.c_double, ctypes.c_int32,
                                           ctypes.c_int32, ctypes.c_float, ctypes.c_int32,
                                           ctypes.c_int32, _i32p, _f32p, _f64p, _f32p]
+        L.dgc_oracle_compress_clip_per_tensor.restype = None
+        L.dgc_oracle_compress_clip_per_tensor.argtypes = [
+            ctypes.c_int32, _i64p, _i64p, _i64p, _i64p, _f32p, _f32p, _f32p, ctypes.c_float,
+            ctypes.c_double, ctypes.c_int32, _f32p, ctypes.c_int32, ctypes.c_int32, _i32p, _f32p,
+            _f64p, _f32p]
         L.dgc_oracle_decode_accumulate.restype = None
         L.dgc_oracle_decode_accumulate.argtypes = [ctypes.c_int32, ctypes.POINTER(_i32p),
                                                    ctypes.POINTER(_f32p), _i64p, _f32p,
@@ -191,6 +196,29 @@ class Worker:
             ctypes.byref(norm),
             ctypes.byref(coef))
         return CompressResult(idx, val, norm.value, np.float32(coef.value))
+
+    def compress_clip_per_tensor(self, g: np.ndarray, coef_override=None,
+                                 brute_force: bool = False):
+        """One iteration with every tensor clipped by its own L2 norm: returns
+        (CompressResult with norm = per-tensor norms, coef = per-tensor coefficients)."""
+        g = _chk(g, np.float32)
+        assert g.size == self.arena_len
+        T = len(self.numel)
+        idx = np.empty(self.nnz, dtype=np.int32)
+        val = np.empty(self.nnz, dtype=np.float32)
+        norms = np.zeros(T, dtype=np.float64)
+        coefs = np.ones(T, dtype=np.float32)
+        ov = None
+        if coef_override is not None:
+            ov = _chk(np.ascontiguousarray(coef_override, dtype=np.float32), np.float32)
+            assert ov.size == T
+        lib().dgc_oracle_compress_clip_per_tensor(
+            T, _p(self.offset, _i64p), _p(self.numel, _i64p), _p(self.k, _i64p),
+            _p(self.out_offset, _i64p), _p(self.u, _f32p), _p(self.v, _f32p), _p(g, _f32p),
+            ctypes.c_float(self.momentum), self.clip_threshold, self.num_workers,
+            None if ov is None else _p(ov, _f32p), int(brute_force), int(self.nesterov),
+            _p(idx, _i32p), _p(val, _f32p), _p(norms, _f64p), _p(coefs, _f32p))
+        return CompressResult(idx, val, norms, coefs)
 
 
 def sample_count(n: int, sample_ratio: float = 0.01) -> int:

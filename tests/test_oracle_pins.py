@@ -278,6 +278,52 @@ def test_clipping_happens_before_accumulation():
     assert w.u[1] == np.float32(0.5) and w.v[1] == np.float32(0.5)
 
 
+def test_clip_per_tensor_option():
+    """Clipping per tensor: each tensor is scaled by thr_local / ||g[j]|| iff its own norm
+    exceeds thr_local; dyadic example by hand, numpy norms, and the difference from the
+    whole-set reading."""
+    # two tensors, N = 4, thr_G = 10 -> thr_local = 5: [6, 8] has norm 10 -> coef 0.5;
+    # [3, 4, 0] has norm 5, not above the threshold -> untouched
+    w = O.Worker([0, 2], [2, 3], 5, 4, 0.0, 10.0, 0.0)          # s = 0: everything is sent
+    g = _f32([6, 8, 3, 4, 0])
+    r = w.compress_clip_per_tensor(g)
+    assert r.norm.tolist() == [10.0, 5.0] and r.coef.tolist() == [0.5, 1.0]
+    assert r.val.tolist() == [3.0, 4.0, 3.0, 4.0, 0.0]
+    # the whole-set reading clips both by one coefficient: norm sqrt(125) > 5
+    w0 = O.Worker([0, 2], [2, 3], 5, 4, 0.0, 10.0, 0.0)
+    r0 = w0.compress(g)
+    assert r0.coef == np.float32(5.0 / np.sqrt(125.0)) and r0.val[2] != 3.0
+    # numpy: per-tensor norms, coefficients and clipped norms on random data with gaps
+    rng = np.random.default_rng(12)
+    numel, offset, L = [1000, 37, 4096], [0, 1024, 1100], 1100 + 4096
+    arena = np.full(L, np.float32(np.nan))
+    scale = [1.0, 0.01, 3.0]
+    for o, n, sc in zip(offset, numel, scale):
+        arena[o:o + n] = (rng.standard_normal(n) * sc).astype(np.float32)
+    w = O.Worker(offset, numel, L, 4, 0.0, 20.0, 0.0)           # thr_local = 10
+    r = w.compress_clip_per_tensor(arena)
+    for j, (o, n) in enumerate(zip(offset, numel)):
+        ref = np.linalg.norm(arena[o:o + n].astype(np.float64))
+        assert abs(r.norm[j] - ref) <= 1e-12 * ref
+        if ref > 10.0:
+            assert abs(np.float64(r.coef[j]) - 10.0 / ref) <= 1e-7 * r.coef[j]
+            sent = r.val[w.out_offset[j]:w.out_offset[j + 1]].astype(np.float64)
+            assert abs(np.linalg.norm(sent) - 10.0) < 1e-5
+        else:
+            assert r.coef[j] == 1.0
+    assert (r.coef < 1).tolist() == [True, False, True]
+    # clipping off: identical to the plain iteration
+    a = O.Worker(offset, numel, L, 4, 0.9, 0.0, 0.99)
+    b = O.Worker(offset, numel, L, 4, 0.9, 0.0, 0.99)
+    ra, rb = a.compress_clip_per_tensor(arena), b.compress(arena)
+    assert ra.idx.tobytes() == rb.idx.tobytes() and ra.val.tobytes() == rb.val.tobytes()
+    assert a.u[:1000].tobytes() == b.u[:1000].tobytes()
+    # the override replaces the computed coefficients
+    c = O.Worker([0, 2], [2, 3], 5, 4, 0.0, 10.0, 0.0)
+    rc = c.compress_clip_per_tensor(g, coef_override=[0.25, 0.5])
+    assert rc.val.tolist() == [1.5, 2.0, 1.5, 2.0, 0.0]
+
+
 # ------------------------------------------------------------------ invariants on a multi-tensor run
 
 def _run_multi(seed, numel, T, momentum, sparsity, clip, workers=4):
