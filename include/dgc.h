@@ -76,6 +76,11 @@ typedef struct dgc_config {
                                      1: Sec. 5 as stated ("paper-literal"): the threshold comes
                                      from the sample, |v| > thr is sent, at most 2 k_j entries
                                      per tensor; the count varies, see dgc_get_nnz             */
+  int32_t        clip_scope;      /* 0: one clipping norm over the worker's whole gradient set
+                                     (Appendix C's ||G^k||_2; the reading used everywhere else).
+                                     1: every tensor is clipped by its own L2 norm against the
+                                     same thr_G * N^-1/2 (Sec. 3.2 speaks of "their L2-norms");
+                                     see dgc_get_clip                                          */
 } dgc_config;
 
 typedef struct dgc_status {
@@ -93,7 +98,7 @@ typedef struct dgc_status {
  * tables.  Synchronous.  The caller's current device is the same after the
  * call as before it.  The state is owned by the caller until
  * dgc_state_destroy.  Errors: DGC_EINVAL (NULL, num_tensors < 1, numel < 1,
- * sparsity outside [0,1), sample_ratio outside [0, 0.5], padded arena >=
+ * sparsity outside [0,1), sample_ratio outside [0, 0.5], select_mode or clip_scope not 0 or 1, padded arena >=
  * 2^31 elements), DGC_ENOMEM, DGC_ECUDA. */
 int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out);
 
@@ -328,6 +333,14 @@ int32_t dgc_get_nnz(dgc_state* st, void* stream, int64_t* total_out, int64_t* pe
  *   kth_key     bit pattern of |v| of the smallest selected entry (the threshold of Algorithm 4)
  *   candidates  entries that passed the sampled threshold (-1: full-selection path taken) */
 int32_t dgc_get_thresholds(dgc_state* st, void* stream, uint32_t* kth_key, int32_t* candidates);
+
+/* Synchronises `stream`, then copies the clipping of the last dgc_compress to host arrays
+ * [num_tensors] (either may be NULL): the L2 norm each tensor was measured by and the coefficient
+ * it was scaled with (Sec. 3.2, Appendix C).  With clip_scope 0 every tensor reports the one
+ * norm and coefficient of the whole set; with clipping off, 0 and 1.  With clip_scope 1,
+ * dgc_status.grad_norm is the norm of the whole set and dgc_status.clip_coef the smallest
+ * coefficient. */
+int32_t dgc_get_clip(dgc_state* st, void* stream, double* norms, float* coefs);
 
 /* Checkpoint / resume: copy u and v (arena_len floats each) to / from host
  * memory.  Synchronous on `stream`.  Either pointer may be NULL. */

@@ -37,7 +37,8 @@ class Config(ctypes.Structure):
                 ("clip_threshold", ctypes.c_float), ("sparsity", ctypes.c_double),
                 ("sample_ratio", ctypes.c_double), ("seed", ctypes.c_uint64),
                 ("device", ctypes.c_int32), ("debug_sample_rank", ctypes.c_int32),
-                ("nesterov", ctypes.c_int32), ("select_mode", ctypes.c_int32)]
+                ("nesterov", ctypes.c_int32), ("select_mode", ctypes.c_int32),
+                ("clip_scope", ctypes.c_int32)]
 
 
 class Status(ctypes.Structure):
@@ -88,6 +89,7 @@ _sigs = {
     "dgc_get_nnz": (ctypes.c_int32, [_vp, _vp, _i64p, _i64p]),
     "dgc_get_status": (ctypes.c_int32, [_vp, _vp, ctypes.POINTER(Status)]),
     "dgc_get_thresholds": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
+    "dgc_get_clip": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_read": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_write": (ctypes.c_int32, [_vp, _vp, _vp, _vp]),
     "dgc_state_set_iterations": (ctypes.c_int32, [_vp, ctypes.c_int64, _vp]),
@@ -148,11 +150,12 @@ class State:
     def __init__(self, tensor_numel: Sequence[int], num_workers: int, momentum: float,
                  clip_threshold: float, sparsity: float, sample_ratio: float = 0.01,
                  seed: int = 0, device: int = 0, debug_sample_rank: int = 0,
-                 nesterov: bool = False, select_mode: int = 0):
+                 nesterov: bool = False, select_mode: int = 0, clip_scope: int = 0):
         numel = (ctypes.c_int64 * len(tensor_numel))(*[int(n) for n in tensor_numel])
         cfg = Config(len(tensor_numel), int(num_workers), numel, float(momentum),
                      float(clip_threshold), float(sparsity), float(sample_ratio), int(seed),
-                     int(device), int(debug_sample_rank), int(bool(nesterov)), int(select_mode))
+                     int(device), int(debug_sample_rank), int(bool(nesterov)), int(select_mode),
+                     int(clip_scope))
         self._h = _vp()
         self.num_tensors = len(tensor_numel)
         self.device = int(device)
@@ -225,6 +228,14 @@ class State:
         _check(_lib.dgc_get_thresholds(self._h, _stream(stream), kth.ctypes.data, cand.ctypes.data),
                "dgc_get_thresholds")
         return kth, cand
+
+    def clip(self, stream=None):
+        """(norms float64[T], coefficients float32[T]) of the last compress call's clipping."""
+        norms = np.zeros(self.num_tensors, np.float64)
+        coefs = np.ones(self.num_tensors, np.float32)
+        _check(_lib.dgc_get_clip(self._h, _stream(stream), norms.ctypes.data, coefs.ctypes.data),
+               "dgc_get_clip")
+        return norms, coefs
 
     def profile_enable(self, max_calls: int) -> None:
         _check(_lib.dgc_profile_enable(self._h, int(max_calls)), "dgc_profile_enable")

@@ -310,6 +310,10 @@ int32_t upload_plan(dgc_state* st, bool first) {
   const size_t o_bstate = o; o = up16(o + NBT * kBigStateWords * 4);
   const size_t o_babove = o; o = up16(o + NBP * 4);
   const size_t o_blast = o; o = up16(o + NBP * kBigLastStride * 4);
+  const bool per_tensor_clip = st->cfg.clip_scope == 1 && st->cfg.clip_threshold > 0.0f;
+  const size_t o_segsq = o; o = up16(o + (per_tensor_clip ? S * 8 : 0));
+  const size_t o_tnorm = o; o = up16(o + T * 8);
+  const size_t o_tcoef = o; o = up16(o + T * 4);
   const size_t bytes = o + 16;
   if (first || bytes > st->d_tables_bytes) {
     if (st->d_tables) dev_free(st, st->d_tables);
@@ -351,6 +355,10 @@ int32_t upload_plan(dgc_state* st, bool first) {
   p.big_state = (int32_t*)(d + o_bstate);
   p.big_above = (int32_t*)(d + o_babove);
   p.big_last = (int32_t*)(d + o_blast);
+  p.clip_scope = per_tensor_clip ? 1 : 0;
+  p.seg_sumsq = (double*)(d + o_segsq);
+  p.t_norm = (double*)(d + o_tnorm);
+  p.t_coef = (float*)(d + o_tcoef);
   p.num_big_parts = (int32_t)NBP; p.num_big_tensors = (int32_t)NBT;
   p.num_tensors = (int32_t)T; p.num_parts = (int32_t)P; p.num_segs = (int32_t)S;
   // candidate lists
@@ -466,6 +474,7 @@ int32_t dgc_state_create(const dgc_config* cfg, dgc_state** out) {
   if (cfg->num_tensors < 1 || !cfg->tensor_numel || cfg->num_workers < 1) return DGC_EINVAL;
   if (!(cfg->sparsity >= 0.0 && cfg->sparsity < 1.0)) return DGC_EINVAL;
   if (cfg->select_mode != 0 && cfg->select_mode != 1) return DGC_EINVAL;
+  if (cfg->clip_scope != 0 && cfg->clip_scope != 1) return DGC_EINVAL;
   if (!(cfg->sample_ratio >= 0.0 && cfg->sample_ratio <= 0.5)) return DGC_EINVAL;
   if (!(cfg->momentum == cfg->momentum)) return DGC_EINVAL;
   int64_t padded = 0;
@@ -596,7 +605,14 @@ static int32_t enqueue_head(dgc_state* st, const float* grad_arena, cudaStream_t
   if (clip) {
     const double thr_local =
         (double)st->cfg.clip_threshold / std::sqrt((double)st->cfg.num_workers);
-    launch(k_sumsq, st->norm_grid, kNormThreads, 0, s, p, grad_arena, thr_local, 1);
+    if (p.clip_scope) {
+      const int grid = (p.num_segs + (kNormThreads / 32) - 1) / (kNormThreads / 32);
+      launch(k_sumsq_segments, grid, kNormThreads, 0, s, p, grad_arena);
+      if ((rc = check_launch()) != DGC_OK) return rc;
+      launch(k_tensor_coef, p.num_tensors, kNormThreads, 0, s, p, thr_local);
+    } else {
+      launch(k_sumsq, st->norm_grid, kNormThreads, 0, s, p, grad_arena, thr_local, 1);
+    }
     if ((rc = check_launch()) != DGC_OK) return rc;
   }
   if (after_norm) DGC_CUDA(cudaEventRecord(after_norm, s));
@@ -1047,6 +1063,22 @@ int32_t dgc_get_status(dgc_state* st, void* stream, dgc_status* out) {
   st->iterations = done;
   const int parity = (int)((st->iterations + 1) & 1);   // parity of the last call
   const bool clip = st->cfg.clip_threshold > 0.0f;
+  if (clip && st->plan.clip_scope) {
+    // per tensor: the norm of the whole set from the tensors' norms, the smallest coefficient
+    const size_t T = st->cfg.num_tensors;
+    std::vector<double> tn(T);
+    std::vector<float> tc(T);
+    DGC_CUDA(cudaMemcpy(tn.data(), st->plan.t_norm, T * 8, cudaMemcpyDeviceToHost));
+    DGC_CUDA(cudaMemcpy(tc.data(), st->plan.t_coef, T * 4, cudaMemcpyDeviceToHost));
+    double ss = 0.0;
+    coef = 1.0f;
+    for (size_t j = 0; j < T; ++j) {
+      ss += tn[j] * tn[j];
+      if (!(tc[j] >= coef)) coef = tc[j];              // (NaN propagates)
+    }
+    norm = done > 0 ? std::sqrt(ss) : 0.0;
+    if (done == 0) coef = 1.0f;
+  }
   out->grad_norm = clip ? norm : 0.0;
   out->clip_coef = clip ? coef : 1.0f;
   out->flags = (int32_t)(diag[parity * 4 + 0] & 0x1F);
@@ -1063,6 +1095,29 @@ int32_t dgc_get_thresholds(dgc_state* st, void* stream, uint32_t* kth_key, int32
   const size_t T = st->cfg.num_tensors;
   if (kth_key) DGC_CUDA(cudaMemcpy(kth_key, st->plan.t_kth, T * 4, cudaMemcpyDeviceToHost));
   if (candidates) DGC_CUDA(cudaMemcpy(candidates, st->plan.t_cand, T * 4, cudaMemcpyDeviceToHost));
+  return DGC_OK;
+}
+
+int32_t dgc_get_clip(dgc_state* st, void* stream, double* norms, float* coefs) {
+  if (!st || !st->alive) return DGC_ESTATE;
+  DGC_CUDA(cudaStreamSynchronize(as_stream(stream)));
+  const size_t T = st->cfg.num_tensors;
+  const bool clip = st->cfg.clip_threshold > 0.0f;
+  if (clip && st->plan.clip_scope) {
+    if (norms) DGC_CUDA(cudaMemcpy(norms, st->plan.t_norm, T * 8, cudaMemcpyDeviceToHost));
+    if (coefs) DGC_CUDA(cudaMemcpy(coefs, st->plan.t_coef, T * 4, cudaMemcpyDeviceToHost));
+    return DGC_OK;
+  }
+  double norm = 0.0;
+  float coef = 1.0f;
+  if (clip) {
+    DGC_CUDA(cudaMemcpy(&norm, st->plan.norm, 8, cudaMemcpyDeviceToHost));
+    DGC_CUDA(cudaMemcpy(&coef, st->plan.coef, 4, cudaMemcpyDeviceToHost));
+  }
+  for (size_t j = 0; j < T; ++j) {
+    if (norms) norms[j] = norm;
+    if (coefs) coefs[j] = coef;
+  }
   return DGC_OK;
 }
 

@@ -133,6 +133,11 @@ struct Plan {
   float* cand_val;
   float* coef;
   double* norm;
+  // clipping per tensor (clip_scope = 1): every tensor by its own norm
+  int32_t clip_scope;
+  double* seg_sumsq;         // [segment] sum of squares of the segment's real elements
+  double* t_norm;            // [tensor] L2 norm of the tensor's gradient
+  float* t_coef;             // [tensor] coefficient applied to it
   double* partials;
   unsigned int* ticket;
   long long* diag;           // [2][4]: flags, full_select, candidates, unused
@@ -431,6 +436,59 @@ k_sumsq(Plan p, const float* __restrict__ g, double thr_local, int clip_on) {
   }
 }
 
+// Clipping per tensor (clip_scope = 1), two launches with a fixed summation order each:
+// k_sumsq_segments: one warp per 512-element segment, fp64 sum of squares of its real elements;
+// k_tensor_coef: one block per tensor folds its segments' sums, writes the tensor's norm and
+// its coefficient thr_local / norm (1 unless the norm exceeds thr_local).
+__global__ void __launch_bounds__(kNormThreads)
+k_sumsq_segments(Plan p, const float* __restrict__ g) {
+  pdl_enter();
+  const int lane = threadIdx.x & 31;
+  const int seg = blockIdx.x * (kNormThreads / 32) + (threadIdx.x >> 5);
+  if (seg >= p.num_segs) return;
+  const float4* g4 = reinterpret_cast<const float4*>(g);
+  const int base = seg * kSeg;
+  float4 x[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) x[i] = __ldg(g4 + (base >> 2) + i * 32 + lane);
+  const int end = __ldg(&p.pm[__ldg(p.seg_part + seg)].end);
+  double acc = 0.0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int e = base + (i * 32 + lane) * 4;
+    if (e + 0 < end) acc += (double)x[i].x * (double)x[i].x;
+    if (e + 1 < end) acc += (double)x[i].y * (double)x[i].y;
+    if (e + 2 < end) acc += (double)x[i].z * (double)x[i].z;
+    if (e + 3 < end) acc += (double)x[i].w * (double)x[i].w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
+  if (lane == 0) p.seg_sumsq[seg] = acc;
+}
+
+__global__ void __launch_bounds__(kNormThreads)
+k_tensor_coef(Plan p, double thr_local) {
+  pdl_enter();
+  __shared__ double swarp[kNormThreads / 32];
+  const int j = blockIdx.x;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const TensorMeta t = load_record(p.tm + j);
+  const int s0 = t.off / kSeg, s1 = (t.end + kSeg - 1) / kSeg;
+  double s = 0.0;
+  for (int i = s0 + threadIdx.x; i < s1; i += kNormThreads) s += __ldcg(p.seg_sumsq + i);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+  if (lane == 0) swarp[warp] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double S = 0.0;
+    for (int w = 0; w < kNormThreads / 32; ++w) S += swarp[w];
+    const double norm = sqrt(S);
+    p.t_norm[j] = norm;
+    p.t_coef[j] = norm > thr_local ? (float)(thr_local / norm) : 1.0f;
+  }
+}
+
 // ------------------------------------------------------------------ K2: sampled threshold proposal
 // Sec. 5: sample |v'| (v' computed on the fly from g, u, v exactly as the main
 // pass will), take the sample's rank-r key as the proposed threshold of the
@@ -474,7 +532,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   {
     const int s = sb.chunk * kSampleThreads + tid;
     if (LITERAL && s < G) {
-      const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
+      const float coef = CLIP ? __ldcg(p.clip_scope ? p.t_coef + j : p.coef) : 1.0f;
       const uint64_t n = (uint64_t)(uint32_t)(t.end - t.off);
       uint32_t karr[4] = {0u, 0u, 0u, 0u};
       uint32_t at[4];
@@ -504,7 +562,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
       have = true;
     } else if (!LITERAL && s < G) {
       const uint32_t W = (uint32_t)((t.end - t.off) >> 2) / (uint32_t)G;   // groups per stratum
-      const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
+      const float coef = CLIP ? __ldcg(p.clip_scope ? p.t_coef + j : p.coef) : 1.0f;
       // stratum s = groups [s*W, (s+1)*W); position inside it from a hash (multiply-high
       // instead of a modulo); the < G groups after the last stratum are never sampled
       const uint32_t h =
@@ -766,7 +824,7 @@ k_update_emit(Plan p, const float* __restrict__ g, float m) {
     const PartMeta pm = load_record(p.pm + part);
     const uint32_t thr = __ldcg(p.p_thr + part);
     const bool tie_on = __ldcg(p.p_tie + part) != 0u;
-    const float coef = CLIP ? __ldcg(p.coef) : 1.0f;
+    const float coef = CLIP ? __ldcg(p.clip_scope ? p.t_coef + pm.tensor : p.coef) : 1.0f;
     const int end = pm.end;
     const bool full = base + kSeg <= end;
     if (p.defer_mask) {

@@ -53,9 +53,10 @@ def test_no_cpu_fallback(B):
 
 
 def test_struct_layout_matches_header(B):
-    # dgc_config: 2 x int32, pointer, 2 x float, 2 x double, uint64, 4 x int32 = 64 bytes
-    assert ctypes.sizeof(B.Config) == 64
-    assert B.Config.nesterov.offset == 56
+    # dgc_config: 2 x int32, pointer, 2 x float, 2 x double, uint64, 5 x int32 (+ 4 bytes of
+    # tail padding to the 8-byte alignment) = 72 bytes
+    assert ctypes.sizeof(B.Config) == 72
+    assert B.Config.nesterov.offset == 56 and B.Config.clip_scope.offset == 64
     assert B.Config.tensor_numel.offset == 8 and B.Config.sparsity.offset == 24
     assert B.Config.seed.offset == 40 and B.Config.device.offset == 48
     assert ctypes.sizeof(B.Status) == 40

@@ -347,6 +347,53 @@ def test_checkpoint_resume_is_bit_identical(P):
     b.close()
 
 
+@pytest.mark.parametrize("workload,nesterov", [("lstm_small", False), ("resnet50", True)])
+def test_clipping_per_tensor_matches_oracle(P, workload, nesterov):
+    """dgc_config.clip_scope = 1: every tensor clipped by its own L2 norm (the oracle's
+    compress_clip_per_tensor).  Norms within 1e-6, coefficients bit for bit (the oracle is re-run
+    with the GPU's coefficients should a last bit differ), then indices, values and state bit
+    for bit; the gradients are scaled so that some tensors exceed the threshold and some do not."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    wl = I.workload(workload)
+    clip, N = 1.0, 4
+    st = B.State(wl.numel, N, wl.momentum, clip, wl.sparsity, seed=11, nesterov=nesterov,
+                 clip_scope=1)
+    L, off = st.arena_len, st.arena_offset
+    cpu = O.Worker(off, wl.numel, L, N, wl.momentum, clip, wl.sparsity, nesterov=nesterov)
+    oi = torch.empty(st.max_nnz, dtype=torch.int32, device="cuda")
+    ov = torch.empty(st.max_nnz, dtype=torch.float32, device="cuda")
+    scale = np.float32(40.0 if workload == "resnet50" else 3.0)
+    overrides, clipped, kept = 0, 0, 0
+    for t in range(3):
+        g = P.arena_with_padding_poison(L, off, wl.numel)
+        I.fill(wl, g, off, worker=2, iteration=t)
+        for o, n in zip(off, wl.numel):
+            g[o:o + n] *= scale
+        st.compress(torch.from_numpy(g).cuda(), oi, ov)
+        norms, coefs = st.clip()
+        status = st.status()
+        snap = (cpu.u.copy(), cpu.v.copy())
+        r = cpu.compress_clip_per_tensor(g)
+        assert np.all(np.abs(norms - r.norm) <= 1e-6 * np.maximum(r.norm, 1e-300))
+        if coefs.tobytes() != r.coef.tobytes():
+            cpu.u[:], cpu.v[:] = snap
+            r = cpu.compress_clip_per_tensor(g, coef_override=coefs)
+            overrides += 1
+        assert oi.cpu().numpy().tobytes() == r.idx.tobytes(), t
+        assert ov.cpu().numpy().tobytes() == r.val.tobytes(), t
+        u, v = st.read()
+        assert u.tobytes() == cpu.u.tobytes() and v.tobytes() == cpu.v.tobytes()
+        assert abs(status.grad_norm - np.sqrt((norms ** 2).sum())) <= 1e-9 * status.grad_norm
+        assert status.clip_coef == coefs.min()
+        clipped += int((coefs < 1).sum())
+        kept += int((coefs == 1).sum())
+    assert clipped > 0 and kept > 0 and overrides <= 1
+    st.close()
+    with pytest.raises(B.DgcError):
+        B.State([100], 1, 0.9, 1.0, 0.9, clip_scope=2)
+
+
 def test_compress_host_matches_device_path(P):
     from paper_1712_01887_b200 import binding as B
     numel = [200000, 3000]
