@@ -229,6 +229,14 @@ void build_host_plan(dgc_state* st, double sparsity) {
     if (sampled) {
       t.key_base = (int32_t)st->sample_keys_total;
       t.chunks = (groups + kSampleThreads - 1) / kSampleThreads;
+      // keys a sampling block keeps for the merge: all `rank` where the sample's key must be
+      // exact (paper-literal mode); otherwise a block's expected share of the tensor's `rank`
+      // largest plus a wide margin (the proposal only has to be safe, see k_sample_threshold)
+      t.rank_local = rank;
+      if (!literal && t.chunks > 1) {
+        const double mu = (double)rank / (double)t.chunks;
+        t.rank_local = std::min(rank, (int)std::ceil(mu + 4.0 * std::sqrt(mu) + 4.0));
+      }
       st->sample_keys_total += 4 * (int64_t)groups;
       for (int c = 0; c < t.chunks; ++c) st->sample_blocks.push_back(SampleBlock{j, c});
     }
@@ -301,6 +309,7 @@ int32_t upload_plan(dgc_state* st, bool first) {
   const size_t o_seg = o; o = up16(o + S * 4);
   const size_t o_samp = o; o = up16(o + NS * sizeof(SampleBlock));
   const size_t o_skeys = o; o = up16(o + (size_t)st->sample_keys_total * 4);
+  const size_t o_sall = o; o = up16(o + (size_t)st->sample_keys_total * 4);
   const size_t o_stick = o; o = up16(o + T * 4);
   const size_t o_scnt = o; o = up16(o + NS * 4);
   const size_t NBP = st->big_parts.size(), NBT = st->big_tensors.size();
@@ -347,6 +356,7 @@ int32_t upload_plan(dgc_state* st, bool first) {
   p.seg_part = (const int32_t*)(d + o_seg);
   p.sample_blocks = (const SampleBlock*)(d + o_samp);
   p.sample_keys = (uint32_t*)(d + o_skeys);
+  p.sample_all = (uint32_t*)(d + o_sall);
   p.sample_ticket = (int32_t*)(d + o_stick);
   p.sample_cnt = (int32_t*)(d + o_scnt);
   p.big_parts = (const int32_t*)(d + o_bparts);

@@ -83,7 +83,9 @@ struct __align__(16) TensorMeta {   // one per tensor, read-only for the kernels
   int32_t key_base, chunks;         // sampling: first key in the sample buffer, blocks that sample
   int32_t big, big_slot;            // big: selected by the multi-block path; slot in its tables
   int32_t samples;                  // paper-literal mode: elements drawn (4 per group, the last
-  int32_t pad_[3];                  // group may be short); otherwise unused
+                                    // group may be short); otherwise unused
+  int32_t rank_local;               // keys each sampling block of the tensor keeps for the merge
+  int32_t pad_[2];
 };
 struct SampleBlock { int32_t tensor, chunk; };   // work item of one k_sample_threshold block
 struct __align__(16) PartMeta {     // one per part (up to kPartSegs segments of one tensor)
@@ -117,7 +119,8 @@ struct Plan {
   int32_t* t_cand;           // per tensor: candidates of the last call, -1 = full selection
   const int32_t* seg_part;   // part of every segment
   const SampleBlock* sample_blocks;
-  uint32_t* sample_keys;     // |v'| keys of the current call's sample, all tensors
+  uint32_t* sample_keys;     // per sampling block: the keys it kept for its tensor's merge
+  uint32_t* sample_all;      // |v'| keys of the current call's whole sample, all tensors
   int32_t* sample_ticket;    // per tensor: sampling blocks that have finished
   int32_t* sample_cnt;       // per sampling block: keys it kept in its slice of sample_keys
   // multi-block selection (tensors with too many candidates for one block)
@@ -526,7 +529,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   const int j = sb.tensor;
   const TensorMeta t = load_record(p.tm + j);
   const int G = t.groups, rank = t.rank;
-  uint4* gkeys = reinterpret_cast<uint4*>(p.sample_keys + t.key_base);
+  uint4* gkeys = reinterpret_cast<uint4*>(p.sample_all + t.key_base);
   uint4 mykeys = make_uint4(0u, 0u, 0u, 0u);
   bool have = false;
   {
@@ -602,7 +605,14 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
     if (tid == 0) { s_cnt = 0; s_max = 0u; }
     __syncthreads();
     uint32_t low = 1u;                             // zeros are never kept: see the union below
-    if (rank <= 4 * nv) {
+    // A block keeps its rank_local largest keys.  With rank_local = rank the union of the
+    // blocks' lists surely holds the tensor's `rank` largest.  The exact mode keeps fewer -- the
+    // share a block can expect of them plus a wide margin -- so that the merge handles a few
+    // hundred keys instead of thousands; should a block have held more of them than that, the
+    // merged key comes out a little low, which only lets a few more candidates through.
+    const int rloc = t.rank_local;
+    if (rloc < rank && have) gkeys[sb.chunk * kSampleThreads + tid] = mykeys;   // (see the merge)
+    if (rloc <= 4 * nv) {
       const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
       if (lane == 0) atomicMax(&s_max, wmax);
       __syncthreads();
@@ -614,7 +624,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
                           f(have, mykeys.z);
                           f(have, mykeys.w);
                         },
-                        rank, 0u, s_max, hist, sh, n_gt_local));
+                        rloc, 0u, s_max, hist, sh, n_gt_local));
     }
     const uint32_t karr[4] = {mykeys.x, mykeys.y, mykeys.z, mykeys.w};
     if (__any_sync(0xFFFFFFFFu, have && tmax >= low)) {
@@ -664,7 +674,10 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
     __syncthreads();
     const int U = s_off[32];
     const uint32_t* keys0 = p.sample_keys + t.key_base;
-    if (U < rank) {
+    bool whole = false;
+    if (U < rank && t.rank_local < rank) {
+      whole = true;      // shortened lists that do not add up to `rank`: select from the whole sample
+    } else if (U < rank) {
       kth = 0u;                                    // fewer than `rank` non-zero keys
       n_eq = 2;                                    // and the zeros beyond them are many
     } else if (U <= kSampleSurvivors) {
@@ -702,7 +715,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
           },
           rank, 0u, 0x7FFFFFFFu, hist, sh, n_gt, &n_eq);
     }
-    done = true;
+    done = !whole;
   }
   if (tid == 0 && !done) { s_cnt = 0; s_max = 0u; }
   __syncthreads();                                    // also orders this block's own key writes

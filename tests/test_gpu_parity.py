@@ -236,6 +236,25 @@ def test_few_distinct_magnitudes_tie_fill_matches_oracle(P, sparsity):
     pair.close()
 
 
+def test_nonzeros_concentrated_in_one_sampling_block(P):
+    """A large tensor whose non-zero entries all lie in its first twentieth: the sampling block
+    of that region holds every one of the sample's largest keys, far more than the shortened
+    list it keeps for the merge, so the merge must notice that the lists do not add up and
+    select from the whole sample instead.  Bit for bit against the oracle, no full selection."""
+    numel = [3_000_000, 70001]
+    pair = P.Pair(numel, 1, 0.9, 0.0, 0.999, seed=21)
+    rep = P.ParityReport()
+    rng = np.random.default_rng(77)
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    for t in range(3):
+        g = P.arena_with_padding_poison(L, off, numel)
+        g[off[0]:off[0] + 150_000] = rng.standard_normal(150_000).astype(np.float32)
+        g[off[1]:off[1] + numel[1]] = rng.standard_normal(numel[1]).astype(np.float32)
+        _, _, st = pair.step(g, rep)
+        assert st.full_select_last == 0 and not st.flags & 2, (t, st.flags)
+    pair.close()
+
+
 def test_forced_full_selection_path_matches(P):
     """debug_sample_rank = 1 proposes the sample maximum: too few pass, every sampled tensor
     falls back to selecting from the whole of v; the result must not change."""
