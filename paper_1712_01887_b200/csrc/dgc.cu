@@ -238,7 +238,12 @@ void build_host_plan(dgc_state* st, double sparsity) {
         t.rank_local = std::min(rank, (int)std::ceil(mu + 4.0 * std::sqrt(mu) + 4.0));
       }
       st->sample_keys_total += 4 * (int64_t)groups;
-      for (int c = 0; c < t.chunks; ++c) st->sample_blocks.push_back(SampleBlock{j, c});
+      for (int c = 0; c < t.chunks; ++c) {
+        SampleBlock sb{};
+        sb.tensor = j;
+        sb.chunk = c;
+        st->sample_blocks.push_back(sb);
+      }
     }
     t.part_first = (int32_t)st->pm.size();
     t.part_num = (int32_t)nparts;
@@ -283,6 +288,7 @@ void build_host_plan(dgc_state* st, double sparsity) {
                    [&](const SampleBlock& a, const SampleBlock& b) {
                      return st->tm[a.tensor].chunks > st->tm[b.tensor].chunks;
                    });
+  for (SampleBlock& sb : st->sample_blocks) sb.t = st->tm[sb.tensor];   // (complete by now)
   st->arena_len = pos;
   st->max_nnz = out;
   st->cand_total = cbase;

@@ -87,7 +87,11 @@ struct __align__(16) TensorMeta {   // one per tensor, read-only for the kernels
   int32_t rank_local;               // keys each sampling block of the tensor keeps for the merge
   int32_t pad_[2];
 };
-struct SampleBlock { int32_t tensor, chunk; };   // work item of one k_sample_threshold block
+struct __align__(16) SampleBlock {   // work item of one k_sample_threshold block: its tensor's
+  TensorMeta t;                      // record travels with it (one round trip instead of two)
+  int32_t tensor, chunk;
+  int32_t pad_[2];
+};
 struct __align__(16) PartMeta {     // one per part (up to kPartSegs segments of one tensor)
   int32_t tensor, end;              // end: arena index one past the part's last real element
   int32_t seg0, nseg;
@@ -307,10 +311,13 @@ __host__ __device__ constexpr int kHistWords(int threads) { return kHistCopies(t
 
 // PRIVATE = false skips the private copies (and the fold with its barrier): for a handful of
 // keys per block the atomics hardly collide and the fixed cost per pass is what counts.
+// max_passes < 4 stops after that many digits and returns the lower edge of the bin that holds
+// the result (a lower bound that at least `rank` keys reach), for callers that only filter.
 template <int THREADS, bool PRIVATE = true, class ForEach>
 __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank, uint32_t base,
                                                       uint32_t maxkey, uint32_t* hist, int* sh,
-                                                      int& n_gt, int* n_eq = nullptr) {
+                                                      int& n_gt, int* n_eq = nullptr,
+                                                      int max_passes = 4) {
   // THREADS = blockDim.x, a compile-time constant so that the slicing below costs no divisions
   constexpr int nt = THREADS;
   const int tid = threadIdx.x;
@@ -328,7 +335,8 @@ __device__ __forceinline__ uint32_t block_select_desc(ForEach for_each, int rank
   }
   __syncthreads();
   int cur = 0;
-  for (int shift = 8 * (passes - 1); shift >= 0; shift -= 8, cur ^= 1) {
+  const int last_shift = 8 * max(passes - max_passes, 0);
+  for (int shift = 8 * (passes - 1); shift >= last_shift; shift -= 8, cur ^= 1) {
     uint32_t* target = PRIVATE ? mine : folded + cur * 256;
     for_each([&](bool valid, uint32_t key) {
       key -= base;
@@ -525,9 +533,9 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   __shared__ uint32_t s_max;
   __shared__ int s_last;
   const int tid = threadIdx.x, lane = tid & 31;
-  const SampleBlock sb = p.sample_blocks[blockIdx.x];
+  const SampleBlock sb = load_record(p.sample_blocks + blockIdx.x);
   const int j = sb.tensor;
-  const TensorMeta t = load_record(p.tm + j);
+  const TensorMeta& t = sb.t;
   const int G = t.groups, rank = t.rank;
   uint4* gkeys = reinterpret_cast<uint4*>(p.sample_all + t.key_base);
   uint4 mykeys = make_uint4(0u, 0u, 0u, 0u);
@@ -624,7 +632,9 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
                           f(have, mykeys.z);
                           f(have, mykeys.w);
                         },
-                        rloc, 0u, s_max, hist, sh, n_gt_local));
+                        rloc, 0u, s_max, hist, sh, n_gt_local, nullptr, 2));
+      // (two digits = 16 bits below the block's largest key: the bound is within 0.4 % of the
+      // block's rloc-th key, the list a few keys longer, the block two radix passes shorter)
     }
     const uint32_t karr[4] = {mykeys.x, mykeys.y, mykeys.z, mykeys.w};
     if (__any_sync(0xFFFFFFFFu, have && tmax >= low)) {
