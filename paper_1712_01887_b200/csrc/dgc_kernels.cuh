@@ -530,7 +530,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   static_assert(kSampleSurvivors <= kHistCopies(kSampleThreads) * 257, "survivors alias the copies");
   __shared__ int sh[3];
   __shared__ int s_cnt;
-  __shared__ uint32_t s_max;
+  __shared__ uint32_t s_max, s_min;
   __shared__ int s_last;
   const int tid = threadIdx.x, lane = tid & 31;
   const SampleBlock sb = load_record(p.sample_blocks + blockIdx.x);
@@ -674,7 +674,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
     // the union of the blocks' slices: counts -> offsets (at most 32 blocks per tensor)
     __shared__ int s_off[33];
     const int first = blockIdx.x - sb.chunk;
-    if (tid == 0) s_max = 0u;
+    if (tid == 0) { s_max = 0u; s_min = 0xFFFFFFFFu; }
     if (tid < 32) {
       const int c = tid < t.chunks ? __ldcg(p.sample_cnt + first + tid) : 0;
       const int incl = warp_incl_scan(c);
@@ -691,7 +691,9 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
       kth = 0u;                                    // fewer than `rank` non-zero keys
       n_eq = 2;                                    // and the zeros beyond them are many
     } else if (U <= kSampleSurvivors) {
-      uint32_t tmax = 0u;
+      // (the lists' keys lie within a factor of a few of each other: selecting between their
+      // smallest and largest key saves the radix pass over the exponent bits they share)
+      uint32_t tmax = 0u, tmin = 0xFFFFFFFFu;
       for (int q = tid >> 5; q < t.chunks; q += kSampleThreads / 32) {
         const int o = s_off[q], c = s_off[q + 1] - o;
         const uint32_t* src = keys0 + q * (4 * kSampleThreads);
@@ -699,20 +701,23 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
           const uint32_t key = __ldcg(src + i);
           surv[o + i] = key;
           tmax = max(tmax, key);
+          tmin = min(tmin, key);
         }
       }
       const uint32_t wmax = __reduce_max_sync(0xFFFFFFFFu, tmax);
-      if (lane == 0) atomicMax(&s_max, wmax);
+      const uint32_t wmin = __reduce_min_sync(0xFFFFFFFFu, tmin);
+      if (lane == 0) { atomicMax(&s_max, wmax); atomicMin(&s_min, wmin); }
       __syncthreads();
+      const uint32_t smin = s_min;
       const int it2 = (U + kSampleThreads - 1) / kSampleThreads;
       kth = block_select_desc<kSampleThreads, false>(
           [&](auto f) {
             for (int it = 0; it < it2; ++it) {
               const int i = it * kSampleThreads + tid;
-              f(i < U, i < U ? surv[i] : 0u);
+              f(i < U, i < U ? surv[i] : smin);
             }
           },
-          rank, 0u, s_max, hist, sh, n_gt, &n_eq);
+          rank, smin, s_max, hist, sh, n_gt, &n_eq);
     } else {
       kth = block_select_desc<kSampleThreads>(
           [&](auto f) {
