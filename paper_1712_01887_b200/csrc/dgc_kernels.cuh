@@ -1902,11 +1902,15 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   const int32_t* cidx = p.cand_idx + pm.cbase;
   const float* cval = p.cand_val + pm.cbase;
   // first kEmitRegs candidates of every thread stay in registers
+  // (values and indices in one round of loads: the index of a candidate that turns out not to
+  // be sent is a wasted word, a dependent second round trip would cost the block's chain more)
   float vals[kEmitRegs];
+  int locs[kEmitRegs];
 #pragma unroll
   for (int b = 0; b < kEmitRegs; ++b) {
     const int i = b * kEmitThreads + tid;
     vals[b] = i < count ? __ldcg(cval + i) : 0.0f;
+    locs[b] = i < count ? __ldcg(cidx + i) : 0;
   }
   // (only the part's own segments: most parts of a many-tensor set are a few segments long)
   for (int i = tid; i < pm.nseg * kMaskStride; i += kEmitThreads) {
@@ -1916,14 +1920,13 @@ k_emit_mask(Plan p, int32_t* __restrict__ out_idx, float* __restrict__ out_val) 
   __syncthreads();
   if (tid == 0) { p.p_count[part] = 0; p.p_eq[part] = 0; }   // ready for the next call
   // mark the candidates that reach the threshold: one bit per element of the part
-  int locs[kEmitRegs];
 #pragma unroll
   for (int b = 0; b < kEmitRegs; ++b) {
     const int i = b * kEmitThreads + tid;
     const uint32_t key = mag_key(vals[b]);
+    const int local = locs[b] - pm.seg0 * kSeg;
     locs[b] = -1;
     if (i < count && key >= kth) {
-      const int local = __ldcg(cidx + i) - pm.seg0 * kSeg;
       locs[b] = local;
       const int word = (local >> 9) * kMaskStride + ((local >> 5) & 15);
       atomicOr((key > kth ? mgt : meq) + word, 1u << (local & 31));
