@@ -1159,7 +1159,7 @@ __device__ __forceinline__ void select_tensor(const Plan& p, int j, const Tensor
       }
     };
     // up to two keys per thread: not worth private histograms
-    if (total <= 2 * THREADS)
+    if (total <= 8 * THREADS)
       kth = block_select_desc<THREADS, false>(each, rank, kbase, kmax, hist, sh, n_gt);
     else
       kth = block_select_desc<THREADS, true>(each, rank, kbase, kmax, hist, sh, n_gt);
