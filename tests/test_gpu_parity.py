@@ -413,6 +413,28 @@ def test_clipping_per_tensor_matches_oracle(P, workload, nesterov):
         B.State([100], 1, 0.9, 1.0, 0.9, clip_scope=2)
 
 
+def test_get_clip_reports_the_whole_set_norm_when_clipping_by_it(P):
+    """dgc_get_clip with the default scope: every tensor reports the one norm and coefficient
+    of the whole set (what dgc_get_status reports); with clipping off, 0 and 1."""
+    from paper_1712_01887_b200 import binding as B
+    numel = [5000, 70001, 64]
+    rng = np.random.default_rng(4)
+    for clip in (1.0, 0.0):
+        st = B.State(numel, 4, 0.9, clip, 0.99, seed=1)
+        L = st.arena_len
+        oi = torch.empty(st.max_nnz, dtype=torch.int32, device="cuda")
+        ov = torch.empty(st.max_nnz, dtype=torch.float32, device="cuda")
+        st.compress(torch.from_numpy(rng.standard_normal(L).astype(np.float32)).cuda(), oi, ov)
+        norms, coefs = st.clip()
+        status = st.status()
+        if clip > 0:
+            assert status.grad_norm > 0.5 and status.clip_coef < 1.0
+            assert (norms == status.grad_norm).all() and (coefs == status.clip_coef).all()
+        else:
+            assert not norms.any() and (coefs == 1.0).all()
+        st.close()
+
+
 def test_compress_host_matches_device_path(P):
     from paper_1712_01887_b200 import binding as B
     numel = [200000, 3000]
