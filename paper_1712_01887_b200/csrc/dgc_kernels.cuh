@@ -528,7 +528,7 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   // selections run without private copies (only the last 512 words of hist are in use)
   uint32_t* surv = hist;
   static_assert(kSampleSurvivors <= kHistCopies(kSampleThreads) * 257, "survivors alias the copies");
-  __shared__ int sh[3];
+  __shared__ int sh[66];
   __shared__ int s_cnt;
   __shared__ uint32_t s_max, s_min;
   __shared__ int s_last;
@@ -604,8 +604,8 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   // instead of re-reading the whole sample.  (If fewer than `rank` keys of the sample are
   // non-zero the union is short and the answer is 0.)
   // (larger ranks: tiny samples, or the large samples of the paper-literal mode, which can also
-  // spread over more blocks than the one warp that scans the blocks' counts covers)
-  const bool local = t.chunks > 1 && t.chunks <= 32 && rank <= kSampleThreads;
+  // spread over more blocks than the one block scan of the blocks' counts covers)
+  const bool local = t.chunks > 1 && t.chunks <= kSampleThreads && rank <= kSampleThreads;
   if (local) {
     uint32_t* slice = p.sample_keys + t.key_base + sb.chunk * (4 * kSampleThreads);
     const int nv = min(kSampleThreads, G - sb.chunk * kSampleThreads);   // threads with a group
@@ -672,17 +672,19 @@ k_sample_threshold(Plan p, const float* __restrict__ g, float m, uint64_t seed_b
   bool done = false;
   if (local) {
     // the union of the blocks' slices: counts -> offsets (at most 32 blocks per tensor)
-    __shared__ int s_off[33];
+    __shared__ int s_off[kSampleThreads + 1];
     const int first = blockIdx.x - sb.chunk;
     if (tid == 0) { s_max = 0u; s_min = 0xFFFFFFFFu; }
-    if (tid < 32) {
+    {
+      // one thread per sampling block of the tensor (at most kSampleThreads of them)
       const int c = tid < t.chunks ? __ldcg(p.sample_cnt + first + tid) : 0;
-      const int incl = warp_incl_scan(c);
-      s_off[tid] = incl - c;
-      if (tid == 31) s_off[32] = incl;
+      int ex, e2, tot, t2;
+      block_excl_scan2(c, 0, sh, ex, e2, tot, t2);
+      if (tid < t.chunks) s_off[tid] = ex;
+      if (tid == 0) s_off[t.chunks] = tot;
     }
     __syncthreads();
-    const int U = s_off[32];
+    const int U = s_off[t.chunks];
     const uint32_t* keys0 = p.sample_keys + t.key_base;
     bool whole = false;
     if (U < rank && t.rank_local < rank) {
