@@ -349,6 +349,12 @@ def measure(args, wl, rank, world, dev, headline):
     c1.record()
     torch.cuda.synchronize()
     compress_ms = c0.elapsed_time(c1) / (K * NW)
+    # what the last of those calls did, per worker: fallbacks would show here
+    last_status = []
+    for s_ in states:
+        q = s_.status()
+        last_status.append({"flags": int(q.flags), "full_select": int(q.full_select_last),
+                            "candidates": int(q.candidates_last)})
 
     # receive side alone: dense decode + SGD (what the step runs) and the fused sparse form
     def _time(fn, reps=20):
@@ -491,7 +497,8 @@ def measure(args, wl, rank, world, dev, headline):
         "compress": {"ms_per_worker": compress_ms, "elements_per_s": total / (compress_ms * 1e-3),
                      "algorithmic_gbs": compress_bytes / (compress_ms * 1e-3) / 1e9,
                      "frac_of_peak": compress_bytes / (compress_ms * 1e-3) / 1e9 / peak,
-                     "what": "one dgc_compress alone on one stream (one worker per GPU)"},
+                     "what": "one dgc_compress alone on one stream (one worker per GPU)",
+                     "last_call_status_per_worker": last_status},
         "step": {"algorithmic_bytes": step_bytes, "algorithmic_gbs": step_gbs,
                  "frac_of_peak": step_gbs / peak},
         "timeline": timeline, "receive": receive, "wire_format": wire, "e2e": e2e,
