@@ -1077,3 +1077,70 @@ def test_timeline_aid_orders_the_kernels_of_a_call(P):
         a.timeline_read()
     a.close()
     b.close()
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_randomised_option_combinations(P, case):
+    """Seeded fuzz over the options that the other tests take one at a time: paper-literal
+    selection with Nesterov momentum and with clipping on or off, per-tensor clipping at every
+    masking and emission mode (with Nesterov or not), each through dgc_compress and through
+    dgc_compress_batch (two workers).  Three iterations, bit for bit against the oracle."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    rng = np.random.default_rng(7000 + case)
+    pool = [1, 513, 8192, 8193, 20000, 70001, 262145, 300000, 524288 + 7, (1 << 21) + 5]
+    numel = [int(x) for x in rng.choice(pool, size=int(rng.integers(2, 5)))]
+    literal = case % 2 == 0
+    nest = bool(rng.integers(0, 2))
+    batch = bool(rng.integers(0, 2))
+    sparsity = float(rng.choice([0.75, 0.9375, 0.99, 0.999]))
+    clip = float(rng.choice([0.0, 1.0])) if literal else 1.0
+    scope = 0 if literal else 1
+    seed, NW = 300 + case, 2
+    sts = [B.State(numel, 4, 0.9, clip, sparsity, seed=seed, nesterov=nest,
+                   select_mode=int(literal), clip_scope=scope) for _ in range(NW)]
+    L, off = sts[0].arena_len, sts[0].arena_offset
+    cpus = [O.Worker(off, numel, L, 4, 0.9, clip, sparsity, nesterov=nest) for _ in range(NW)]
+    cap = sts[0].max_nnz
+    oi = [torch.empty(cap, dtype=torch.int32, device="cuda") for _ in range(NW)]
+    ov = [torch.empty(cap, dtype=torch.float32, device="cuda") for _ in range(NW)]
+    for t in range(3):
+        gs = []
+        for w in range(NW):
+            g = P.arena_with_padding_poison(L, off, numel)
+            for o, n in zip(off, numel):
+                scale = 10.0 ** float(rng.integers(-2, 2))       # some tensors clipped, some not
+                g[o:o + n] = (rng.standard_normal(n) * scale).astype(np.float32)
+            gs.append(g)
+        dev = [torch.from_numpy(g).cuda() for g in gs]
+        if batch:
+            B.compress_batch(sts, dev, oi, ov)
+        else:
+            for w in range(NW):
+                sts[w].compress(dev[w], oi[w], ov[w])
+        for w in range(NW):
+            status = sts[w].status()
+            snap = (cpus[w].u.copy(), cpus[w].v.copy())
+            if literal:
+                r, nnz = O.compress_sampled(cpus[w], gs[w], seed=seed, iteration=t)
+                if np.float32(status.clip_coef).tobytes() != np.float32(r.coef).tobytes():
+                    cpus[w].u[:], cpus[w].v[:] = snap
+                    r, nnz = O.compress_sampled(cpus[w], gs[w], seed=seed, iteration=t,
+                                                coef_override=status.clip_coef)
+                total, per = sts[w].nnz()
+                assert per.tolist() == nnz.tolist(), (case, t, w)
+            else:
+                norms, coefs = sts[w].clip()
+                r = cpus[w].compress_clip_per_tensor(gs[w])
+                assert np.all(np.abs(norms - r.norm) <= 1e-6 * np.maximum(r.norm, 1e-300))
+                if coefs.tobytes() != r.coef.tobytes():
+                    cpus[w].u[:], cpus[w].v[:] = snap
+                    r = cpus[w].compress_clip_per_tensor(gs[w], coef_override=coefs)
+                total = cap
+            assert total == r.idx.size, (case, t, w)
+            assert oi[w][:total].cpu().numpy().tobytes() == r.idx.tobytes(), (case, t, w)
+            assert ov[w][:total].cpu().numpy().tobytes() == r.val.tobytes(), (case, t, w)
+    for w in range(NW):
+        u, v = sts[w].read()
+        assert u.tobytes() == cpus[w].u.tobytes() and v.tobytes() == cpus[w].v.tobytes(), (case, w)
+        sts[w].close()
