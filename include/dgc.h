@@ -245,8 +245,8 @@ int32_t dgc_decode_rejected(int32_t num_workers, int64_t dense_len, const void* 
  * must not exceed DGC_STATIC_DECODE_WORDS (e.g. 8 workers up to 130 M dense elements); a
  * larger problem returns DGC_ECAPACITY and enqueues nothing.
  *   The first call on each device looks up the array's device address (the device that is
- * current at that call must be the one that owns the buffers); make that first call before
- * starting any stream capture.  All calls on a device share the one array: it still holds the
+ * current at that call must be the one that owns the buffers).  All calls on a device share
+ * the one array: it still holds the
  * previous call's boundaries, which is harmless because every word a call reads it has first
  * written itself, but two calls whose kernels overlap on the GPU (different streams, no
  * ordering) race on it and give undefined results.  Asynchronous on `stream`. */
