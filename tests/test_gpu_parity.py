@@ -1144,3 +1144,62 @@ def test_randomised_option_combinations(P, case):
         u, v = sts[w].read()
         assert u.tobytes() == cpus[w].u.tobytes() and v.tobytes() == cpus[w].v.tobytes(), (case, w)
         sts[w].close()
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_randomised_wide(P, case):
+    """A wider seeded fuzz: 1 to 7 tensors of sizes around every boundary (up to 2^23 elements),
+    every sparsity the schedule and the sweeps use and the switch points between them, momentum
+    0 to 0.99, 1 to 64 workers in the clip scale, sample ratios 0.1 % to 50 %, sparsity changed
+    between iterations, and values that are denormal, near the fp32 maximum (sums overflow to
+    Inf, Inf - Inf gives NaN) or infinite.  Indices bit for bit; values and state bit for bit
+    with a NaN matching any NaN."""
+    rng = np.random.default_rng(90000 + case)
+    pool = [1, 2, 3, 4, 5, 31, 32, 33, 511, 512, 513, 1023, 4096, 8191, 8192, 8193, 8704, 16385,
+            20000, 65536, 70001, 131073, 262143, 262144, 262145, 300000, 524288, 524289, 786433,
+            1 << 20, (1 << 21) + 5, 3000000, 4194304 + 1, 6000000]
+    numel = [int(x) for x in rng.choice(pool, size=int(rng.integers(1, 7)))]
+    if case % 7 == 0:
+        numel.append(1 << 23)
+    sparsity = float(rng.choice([0.0, 0.25, 0.5, 0.75, 0.8749, 0.875, 0.9, 0.9375, 0.984375, 0.99,
+                                 0.996, 0.999, 0.9999, 0.99999]))
+    clip = float(rng.choice([0.0, 0.3, 1.0, 1e6]))
+    pair = P.Pair(numel, int(rng.choice([1, 2, 8, 64])), float(rng.choice([0.0, 0.5, 0.9, 0.99])),
+                  clip, sparsity, seed=int(rng.integers(1, 1 << 30)),
+                  nesterov=bool(rng.integers(0, 2)),
+                  sample_ratio=float(rng.choice([0.001, 0.003, 0.01, 0.05, 0.5])))
+    rep = P.ParityReport()
+    off, L = pair.gpu.arena_offset, pair.gpu.arena_len
+    kinds = ["normal", "student", "sparse", "levels", "const", "zero", "denorm", "huge", "special"]
+    iters = int(rng.integers(2, 6))
+    for t in range(iters):
+        if t > 0 and rng.random() < 0.3:
+            pair.set_sparsity(float(rng.choice([0.5, 0.75, 0.9375, 0.99, 0.999, 0.9999])))
+        g = P.arena_with_padding_poison(L, off, numel)
+        for o, n in zip(off, numel):
+            kind = kinds[int(rng.integers(0, len(kinds)))]
+            if kind == "normal":
+                x = rng.standard_normal(n)
+            elif kind == "student":
+                x = rng.standard_t(2, size=n) * 1e-4
+            elif kind == "sparse":
+                x = rng.standard_normal(n) * (rng.random(n) < 0.003)
+            elif kind == "levels":
+                x = rng.integers(-2, 3, size=n) * 0.125
+            elif kind == "const":
+                x = np.full(n, 0.5) * (rng.integers(0, 2, size=n) * 2 - 1)
+            elif kind == "denorm":
+                x = rng.standard_normal(n) * 1e-41
+            elif kind == "huge":
+                x = rng.standard_normal(n) * 1e30
+            elif kind == "special":
+                x = rng.standard_normal(n)
+                if clip == 0.0 and n > 8:
+                    m = rng.integers(0, n, size=2)
+                    x[m[0]], x[m[1]] = np.inf, -np.inf
+            else:
+                x = np.zeros(n)
+            with np.errstate(over="ignore"):
+                g[o:o + n] = x.astype(np.float32)
+        pair.step(g, rep, check_state=(t == iters - 1))
+    pair.close()
