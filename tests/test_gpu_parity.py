@@ -1203,3 +1203,52 @@ def test_randomised_wide(P, case):
                 g[o:o + n] = x.astype(np.float32)
         pair.step(g, rep, check_state=(t == iters - 1))
     pair.close()
+
+
+@pytest.mark.parametrize("case", range(16))
+def test_randomised_receive_side_and_wire_format(P, case):
+    """Seeded fuzz of the receive side: 1 to 64 workers, dense lengths around the 4096-element
+    tile and up to 5 Mi, lists from empty to complete, values denormal to near the fp32 maximum
+    (sums overflow).  Decode, SGD, the fused sparse and the one-pass forms through
+    parity_util.receive_side; the workspace-free decode where its limit allows; the run-length
+    wire format of one list, encoded and decoded, against the oracle's."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    rng = np.random.default_rng(50000 + case)
+    N = int(rng.choice([1, 2, 3, 4, 8, 17, 64]))
+    L = int(rng.choice([1, 2, 511, 4095, 4096, 4097, 8192, 100000, 262144, 1 << 20, 3000001,
+                        5 << 20]))
+    il, vl = [], []
+    for w in range(N):
+        dens = float(rng.choice([0.0, 1e-5, 1e-3, 0.01, 0.25, 1.0]))
+        m = int(min(L, rng.binomial(L, dens))) if dens < 1.0 else L
+        idx = (np.sort(rng.choice(L, size=m, replace=False)).astype(np.int32) if m < L
+               else np.arange(L, dtype=np.int32))
+        kind = int(rng.integers(0, 4))
+        val = (rng.standard_normal(m) * [1.0, 1e-41, 1e30][kind] if kind < 3
+               else rng.integers(-2, 3, size=m) * 0.5)
+        with np.errstate(over="ignore"):
+            il.append(idx)
+            vl.append(val.astype(np.float32))
+    w0 = rng.standard_normal(L).astype(np.float32)
+    ref, _ = P.receive_side(il, vl, L, w0, float(rng.choice([0.0, 0.1, 1.0, 1e-3])))
+    if N * ((L + 4095) // 4096 + 1025) <= B.STATIC_DECODE_WORDS:
+        di = [torch.from_numpy(a).cuda() for a in il]
+        dv = [torch.from_numpy(a).cuda() for a in vl]
+        dense = torch.full((L,), float("nan"), dtype=torch.float32, device="cuda")
+        B.decode_accumulate_static(di, dv, dense)
+        P._assert_bits(dense.cpu().numpy(), ref, "workspace-free decode")
+        assert B.decode_rejected(N, L) == 0
+    for idx, val in zip(il, vl):
+        if idx.size == 0:
+            continue
+        runs, values = B.encode_runlength(torch.from_numpy(idx).cuda(),
+                                          torch.from_numpy(val).cuda(), L)
+        ro, vo = O.encode_runlength(idx, val, B.runlength_max_entries(idx.size, L))
+        assert runs.cpu().numpy().tobytes() == ro.tobytes()
+        P._assert_bits(values.cpu().numpy(), vo, "run-length values")
+        i2, v2, _ = B.decode_runlength(runs, values)
+        io, vo2 = O.decode_runlength(ro, vo)
+        assert i2.cpu().numpy().tobytes() == io.tobytes()
+        P._assert_bits(v2.cpu().numpy(), vo2, "run-length decoded values")
+        break
