@@ -1252,3 +1252,65 @@ def test_randomised_receive_side_and_wire_format(P, case):
         assert i2.cpu().numpy().tobytes() == io.tobytes()
         P._assert_bits(v2.cpu().numpy(), vo2, "run-length decoded values")
         break
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_randomised_paper_literal_selection(P, case):
+    """Seeded fuzz of select_mode = 1 (Sec. 5 as stated): tensor sizes from 1 element to 2^23,
+    sample ratios 0.1 % to 10 %, sparsities 50 % to 99.99 %, momentum, Nesterov and clipping on or
+    off, value distributions with ties, zeros and heavy tails.  Per-tensor counts, indices, values
+    and state bit for bit against the oracle, which draws the same positions from the same
+    counter-based generator."""
+    from oracle import dgc_oracle as O
+    from paper_1712_01887_b200 import binding as B
+    rng = np.random.default_rng(30000 + case)
+    pool = [1, 2, 3, 5, 31, 512, 513, 4096, 8192, 8193, 20000, 70001, 262144, 262145, 300000,
+            524289, 1 << 20, (1 << 21) + 5, 3000000]
+    numel = [int(x) for x in rng.choice(pool, size=int(rng.integers(1, 6)))]
+    if case % 9 == 0:
+        numel.append(int(rng.choice([1 << 22, 6000000, (1 << 23) + 5])))
+    sparsity = float(rng.choice([0.5, 0.75, 0.9375, 0.99, 0.996, 0.999, 0.9999]))
+    ratio = float(rng.choice([0.001, 0.002, 0.01, 0.03, 0.1]))
+    clip = float(rng.choice([0.0, 1.0]))
+    nest = bool(rng.integers(0, 2))
+    mom = float(rng.choice([0.0, 0.9]))
+    seed = int(rng.integers(1, 1 << 40))
+    st = B.State(numel, 4, mom, clip, sparsity, seed=seed, select_mode=1, sample_ratio=ratio,
+                 nesterov=nest)
+    L, off = st.arena_len, st.arena_offset
+    cpu = O.Worker(off, numel, L, 4, mom, clip, sparsity, nesterov=nest)
+    oi = torch.empty(st.max_nnz, dtype=torch.int32, device="cuda")
+    ov = torch.empty(st.max_nnz, dtype=torch.float32, device="cuda")
+    kinds = ["normal", "student", "sparse", "levels", "const", "zero"]
+    for t in range(int(rng.integers(2, 5))):
+        g = P.arena_with_padding_poison(L, off, numel)
+        for o, n in zip(off, numel):
+            kind = kinds[int(rng.integers(0, len(kinds)))]
+            if kind == "normal":
+                x = rng.standard_normal(n)
+            elif kind == "student":
+                x = rng.standard_t(2, size=n) * 1e-4
+            elif kind == "sparse":
+                x = rng.standard_normal(n) * (rng.random(n) < 0.003)
+            elif kind == "levels":
+                x = rng.integers(-2, 3, size=n) * 0.125
+            elif kind == "const":
+                x = np.full(n, 0.5) * (rng.integers(0, 2, size=n) * 2 - 1)
+            else:
+                x = np.zeros(n)
+            g[o:o + n] = x.astype(np.float32)
+        st.compress(torch.from_numpy(g).cuda(), oi, ov)
+        status = st.status()
+        total, per = st.nnz()
+        snap = (cpu.u.copy(), cpu.v.copy())
+        r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t, sample_ratio=ratio)
+        if np.float32(status.clip_coef).tobytes() != np.float32(r.coef).tobytes():
+            cpu.u[:], cpu.v[:] = snap
+            r, nnz = O.compress_sampled(cpu, g, seed=seed, iteration=t, sample_ratio=ratio,
+                                        coef_override=status.clip_coef)
+        assert per.tolist() == nnz.tolist(), (case, t, numel, sparsity, ratio)
+        assert oi[:total].cpu().numpy().tobytes() == r.idx.tobytes(), (case, t)
+        assert ov[:total].cpu().numpy().tobytes() == r.val.tobytes(), (case, t)
+    u, v = st.read()
+    assert u.tobytes() == cpu.u.tobytes() and v.tobytes() == cpu.v.tobytes()
+    st.close()
