@@ -1314,3 +1314,40 @@ def test_randomised_paper_literal_selection(P, case):
     u, v = st.read()
     assert u.tobytes() == cpu.u.tobytes() and v.tobytes() == cpu.v.tobytes()
     st.close()
+
+
+def test_host_buffer_calls_follow_sparsity_changes(P):
+    """dgc_compress_host and dgc_compress_host_batch across dgc_set_sparsity in both directions
+    (their device staging must grow with the list length): bit for bit what dgc_compress gives
+    on device buffers, lists and final state."""
+    from paper_1712_01887_b200 import binding as B
+    numel = [300000, 70001, 64, 9000, 600000]
+    NW = 3
+    rng = np.random.default_rng(5)
+    dev = [B.State(numel, NW, 0.9, 1.0, 0.999, seed=w) for w in range(NW)]
+    host = [B.State(numel, NW, 0.9, 1.0, 0.999, seed=w) for w in range(NW)]
+    L = dev[0].arena_len
+    for t, s in enumerate([0.999, 0.75, 0.75, 0.9999, 0.5, 0.999, 0.99]):
+        for st in dev + host:
+            st.set_sparsity(s)
+        nnz = dev[0].max_nnz
+        hi = [torch.empty(nnz, dtype=torch.int32).pin_memory() for _ in range(NW)]
+        hv = [torch.empty(nnz, dtype=torch.float32).pin_memory() for _ in range(NW)]
+        gh = [torch.from_numpy(rng.standard_normal(L).astype(np.float32)).pin_memory()
+              for _ in range(NW)]
+        if t % 2 == 0:
+            B.compress_host_batch(host, gh, hi, hv)
+        else:
+            for w in range(NW):
+                host[w].compress_host(gh[w], hi[w], hv[w])
+        for w in range(NW):
+            oi = torch.empty(nnz, dtype=torch.int32, device="cuda")
+            ov = torch.empty(nnz, dtype=torch.float32, device="cuda")
+            dev[w].compress(gh[w].cuda(), oi, ov)
+            assert torch.equal(oi.cpu(), hi[w]), (t, w)
+            assert torch.equal(ov.cpu().view(torch.int32), hv[w].view(torch.int32)), (t, w)
+    for w in range(NW):
+        a, b = dev[w].read(), host[w].read()
+        assert a[0].tobytes() == b[0].tobytes() and a[1].tobytes() == b[1].tobytes()
+        dev[w].close()
+        host[w].close()
