@@ -213,7 +213,10 @@ int32_t dgc_compress_host_batch(int32_t num_states, dgc_state* const* states,
  * dense_out or the workspace or read outside the lists: pairs that do not
  * belong where the order puts them are skipped, the sums of the affected
  * entries are then unspecified, and dgc_decode_rejected reports how many pairs
- * were at fault.  1 <= num_workers <= DGC_MAX_DECODE_WORKERS.  Asynchronous on
+ * were at fault.  Such a list can also make the call slow: the work grows with
+ * the sum of the upward index jumps between consecutive pairs, which is at most
+ * dense_len for an ascending list but up to nnz * dense_len / 4096 steps for
+ * arbitrary data.  1 <= num_workers <= DGC_MAX_DECODE_WORKERS.  Asynchronous on
  * `stream`. */
 int32_t dgc_decode_accumulate(int32_t num_workers, const int32_t* const* idx_lists,
                               const float* const* val_lists, const int64_t* nnz, float* dense_out,
